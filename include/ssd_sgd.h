@@ -1,0 +1,245 @@
+/*
+ * ssd_sgd.h - C ABI of the SSD-SGD update path on one NVIDIA B200 (sm_100a).
+ *
+ * SSD-SGD ("Several Steps Delay SGD", arXiv 2012.05396) trains with a
+ * parameter server that applies a synchronous momentum-SGD update from the
+ * gradients of K workers at every iteration, while each worker pulls the global
+ * weight only once every k iterations and, in between, advances a local copy of
+ * the weights with the GLU rule ("global gradient for local update").  This
+ * library is the per-iteration parameter-update arithmetic of that method over
+ * the flattened model state.  The K workers are K sets of buffers in one GPU's
+ * memory: a "push" is the server kernel reading worker i's gradient buffer, a
+ * "pull" is a store of the global weight into worker i's local weight.
+ *
+ * Conventions
+ *  - Every pointer in ssd_buffers and every gradient pointer is DEVICE memory
+ *    owned by the caller, 16-byte aligned, holding at least ssd_arena_numel()
+ *    elements.  The library never allocates, frees or retains device memory of
+ *    its own; a context holds host-side metadata only.  Pointer *tables*
+ *    (w_loc, pre, w_dev, grads) are HOST arrays of K device pointers and are
+ *    copied when passed.
+ *  - State is float32.  Gradients are float32 or bfloat16 (widened exactly).
+ *  - Arithmetic: IEEE-754 binary32, round to nearest even, every multiply and
+ *    add rounded separately (no fused multiply-add), operands in the order
+ *    written below, the K gradients summed left to right (worker 0 first).
+ *    Results are therefore unique and reproducible bit for bit.
+ *  - Calls only enqueue work on `cuda_stream` (a cudaStream_t passed as void*,
+ *    NULL = the legacy default stream) and return; they never synchronise.
+ *    Work of successive calls on the same stream is ordered by the stream.
+ *  - Every call returns an ssd_status.  Arguments are validated before any
+ *    launch; on an error nothing was enqueued and no counter moved.
+ *  - A context is not thread-safe; use one per host thread or lock around it.
+ *
+ * Arena layout.  A parameter layout is an ordered list of T tensors given by
+ * their element counts.  Tensor t lives at element offset ssd_tensor_offset(t)
+ * of every buffer; offsets are multiples of 4 elements (16 bytes in float32),
+ * the gaps are padding that the update treats like any other element (keep
+ * them zero).  All kernels sweep the arena as one flat stream.
+ *
+ * Schedule (Algorithm 1 and Algorithm 2 of the paper).  Iteration n = 0,1,...
+ *   warm-up   n < W, or delay_k == 0: plain synchronous SGD; workers compute on
+ *             the global weight.  On the last warm-up iteration (n == W-1) each
+ *             worker keeps a copy of the new global weight as its local weight
+ *             (SSD_FLAG_COPY).  W counts iterations: the paper's loop
+ *             "while num <= wp" runs W = wp+1 times.
+ *   delay     d = n - W >= 0.  Every iteration: server update, then one GLU
+ *             update per worker.  SSD_FLAG_FIRST on d == 0 (pre_weight is
+ *             initialised with the local weight), SSD_FLAG_REFRESH when d > 0
+ *             and d % k == 0 (pre_weight is overwritten, Algorithm 2),
+ *             SSD_FLAG_PULL when d % k == k-1 (Algorithm 1).  These tests equal
+ *             the printed ones, num % k == k-1 and loc_update % k == 0, whenever
+ *             the paper's own constraint (1+wp) % k == 0 holds, and stay well
+ *             defined when it does not.
+ */
+#ifndef SSD_SGD_H
+#define SSD_SGD_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ssd_ctx ssd_ctx;
+
+typedef enum {
+    SSD_OK = 0,
+    SSD_ERR_ARG = 1,      /* NULL pointer, value out of range, unknown enum   */
+    SSD_ERR_ALIGN = 2,    /* a device pointer is not 16-byte aligned          */
+    SSD_ERR_LAYOUT = 3,   /* empty or oversized layout, negative element count */
+    SSD_ERR_STATE = 4,    /* call not valid in the context's current stage    */
+    SSD_ERR_CUDA = 5,     /* the CUDA runtime reported an error on launch     */
+    SSD_ERR_NOMEM = 6     /* host allocation of the context failed            */
+} ssd_status;
+
+typedef enum { SSD_F32 = 0, SSD_BF16 = 1 } ssd_dtype;
+
+enum { SSD_STAGE_WARMUP = 0, SSD_STAGE_DELAY = 1 };
+enum { SSD_FLAG_FIRST = 1, SSD_FLAG_REFRESH = 2, SSD_FLAG_PULL = 4, SSD_FLAG_COPY = 8 };
+enum { SSD_VIEW_GLOBAL = 0, SSD_VIEW_LOCAL = 1, SSD_VIEW_DEVICE = 2 };
+
+#define SSD_MAX_WORKERS 32
+
+/* Parameter layout: element counts of the T tensors (host array, copied). */
+typedef struct {
+    int32_t num_tensors;          /* T >= 1                                    */
+    const int64_t *numel;         /* numel[t] >= 0; sum of padded counts < 2^40 */
+} ssd_layout;
+
+/* Hyper-parameters (Table 1 of the paper) and the schedule inputs of Algorithm 1. */
+typedef struct {
+    int32_t K;                    /* workers, 1..SSD_MAX_WORKERS                */
+    float lr;                     /* server learning rate, > 0                  */
+    float momentum;               /* m, 0 <= m < 1                              */
+    float wd;                     /* weight decay, used by server and GLU       */
+    int32_t warmup_iters;         /* W >= 0, number of SSGD iterations (wp + 1) */
+    int32_t delay_k;              /* k >= 0; 0 = synchronous SGD forever        */
+    float lr_local;               /* GLU learning rate; NaN = 4 * lr (Section 4.1) */
+    float alpha;                  /* weight of the local gradient; NaN = 2.0    */
+    float beta;                   /* weight of grad_sync; NaN = 0.5             */
+    float rescale;                /* factor on the K-sum; NaN = 1/K (average)   */
+    int32_t grad_dtype;           /* ssd_dtype of every gradient buffer         */
+} ssd_hparams;
+
+/* Caller-owned device state.  w_loc, pre, w_dev: host arrays of K device pointers.
+ * The K*3+2 buffers must not overlap each other or any gradient buffer. */
+typedef struct {
+    float *w;                     /* global weight w_t (server)                 */
+    float *mom;                   /* server momentum mom_t                      */
+    float *const *w_loc;          /* local weight w'_{t,i} of each worker       */
+    float *const *pre;            /* pre_weight of each worker                  */
+    float *const *w_dev;          /* device weights of each worker; written only
+                                     on pull iterations (see ssd_worker_weights) */
+} ssd_buffers;
+
+/* Arena length in elements for a layout: the sum of the element counts, each
+ * rounded up to a multiple of 4.  Needs no context.  Errors: SSD_ERR_ARG (NULL),
+ * SSD_ERR_LAYOUT. */
+ssd_status ssd_arena_numel(const ssd_layout *layout, int64_t *padded_numel);
+
+/* Creates a context.  Copies the layout, resolves NaN hyper-parameters to the
+ * paper's defaults and derives, in double precision from the float-typed
+ * hyper-parameters with one final rounding to float,
+ *     c       = (1 - m) / (lr * k)      the grad_sync scale of Section 3.3
+ *     rescale = 1 / K                   when averaging.
+ * Does not touch any buffer.  Before the first step the caller sets w = w_0,
+ * mom = 0 and, when warmup_iters == 0, also w_loc[i] = w_0 for every worker
+ * (Algorithm 1 starts by pulling w_0); ssd_broadcast_weights does the latter.
+ * Errors: SSD_ERR_ARG, SSD_ERR_ALIGN, SSD_ERR_LAYOUT, SSD_ERR_NOMEM, and
+ * SSD_ERR_CUDA when no CUDA device is usable.  *out is NULL on error. */
+ssd_status ssd_init(ssd_ctx **out, const ssd_layout *layout, const ssd_hparams *hp,
+                    const ssd_buffers *buffers);
+
+/* Releases the context (host memory only).  NULL is accepted. */
+void ssd_destroy(ssd_ctx *ctx);
+
+/* Element offset of tensor `tensor` in every arena. */
+ssd_status ssd_tensor_offset(const ssd_ctx *ctx, int32_t tensor, int64_t *elem_offset);
+
+/* Stage and flags of iteration `iter` under the context's W and k (pure function
+ * of its arguments and the two schedule inputs; see "Schedule" above). */
+ssd_status ssd_schedule(const ssd_ctx *ctx, int64_t iter, int32_t *stage, int32_t *flags);
+
+/* Server side of one iteration (Eq. 6 with momentum, Section 3.2.1): for every
+ * arena element j
+ *     s    = ((g_0[j] + g_1[j]) + g_2[j]) + ... + g_{K-1}[j]
+ *     grad = s * rescale
+ *     mom[j] = m * mom[j] - lr * (grad + wd * w[j])
+ *     w[j]   = w[j] + mom[j]
+ * `grads`: host array of K device pointers (dtype = grad_dtype), read only.
+ * Does not read or move the context's counters: it is the whole of synchronous
+ * SGD when used alone.  One kernel launch. */
+ssd_status ssd_server_sync_update(ssd_ctx *ctx, const void *const *grads, void *cuda_stream);
+
+/* One GLU call of worker `worker` (Algorithm 2 and the GLU rule of Section
+ * 3.2.1, with the descent sign that the server rule and grad_sync imply):
+ *     if FIRST:   pre_i[j] = w_loc_i[j]
+ *     gs = (pre_i[j] - w_loc_i[j]) * c
+ *     if REFRESH: pre_i[j] = w_loc_i[j]                (value before the update)
+ *     r  = w_loc_i[j] - lr_local * ((alpha * g_i[j] + wd * w_loc_i[j]) + beta * gs)
+ *     if PULL:    w_dev_i[j] = r ; w_loc_i[j] = w[j]   (Algorithm 1: the devices keep
+ *                 the GLU result, the local weight takes the pulled global weight)
+ *     else:       w_loc_i[j] = r
+ * `flags` is any combination of SSD_FLAG_FIRST / REFRESH / PULL.  With PULL, `w`
+ * must already hold this iteration's server result (enqueue the server update
+ * first on the same stream).  Does not read or move the counters.  Errors:
+ * SSD_ERR_ARG (worker out of range, unknown flag, NULL grad), SSD_ERR_STATE
+ * (delay_k == 0: there is no delay stage), SSD_ERR_ALIGN.  One kernel launch. */
+ssd_status ssd_worker_glu_update(ssd_ctx *ctx, int32_t worker, const void *grad, int32_t flags,
+                                 void *cuda_stream);
+
+/* Body of Algorithm 1 for one worker at the context's current iteration, to be
+ * enqueued after ssd_server_sync_update of the same iteration: in the warm-up
+ * stage it stores w into w_loc_i on the last warm-up iteration and does nothing
+ * otherwise (`grad` may be NULL there); in the delay stage it is
+ * ssd_worker_glu_update with the flags of ssd_schedule.  Does not move the
+ * counters: call ssd_advance once all K workers are enqueued. */
+ssd_status ssd_worker_local_step(ssd_ctx *ctx, int32_t worker, const void *grad, void *cuda_stream);
+
+/* Ends an iteration assembled from the two calls above: iter += 1 and, in the
+ * delay stage, loc_update += 1. */
+ssd_status ssd_advance(ssd_ctx *ctx);
+
+/* One whole iteration for the server and all K workers, then ssd_advance.  Same
+ * results, bit for bit, as ssd_server_sync_update + K * ssd_worker_local_step,
+ * but as ONE fused kernel in which every gradient element is read once and
+ * feeds both the server sum and its own worker's GLU update (the paper notes
+ * that push and local update only read the gradient, Section 2.2). */
+ssd_status ssd_step(ssd_ctx *ctx, const void *const *grads, void *cuda_stream);
+
+/* ssd_step for gradients that arrive in HOST memory (as they would from a
+ * network push).  `host_grads`: K host pointers (pinned memory for asynchronous
+ * copies); `staging`: K device buffers of arena size (gradient dtype) that
+ * receive them; `host_w_out`: optional host buffer that receives the new global
+ * weight w (NULL = no read-back).  Enqueues K host-to-device copies, the step and
+ * the device-to-host copy on `cuda_stream`; the caller synchronises the stream
+ * before reading host_w_out or reusing host_grads. */
+ssd_status ssd_step_host(ssd_ctx *ctx, const void *const *host_grads, void *const *staging,
+                         float *host_w_out, void *cuda_stream);
+
+/* w_loc[i] = w for every worker (the initial pull of Algorithm 1).  Needed before
+ * the first step only when warmup_iters == 0.  One kernel launch. */
+ssd_status ssd_broadcast_weights(ssd_ctx *ctx, void *cuda_stream);
+
+/* Where worker `worker` finds the weights for its next forward/backward pass
+ * after the iterations done so far: the global w in the warm-up stage, w_loc_i
+ * after a GLU step without pull, w_dev_i after a pull iteration.  `view`
+ * receives the SSD_VIEW_* code; either output may be NULL. */
+ssd_status ssd_worker_weights(const ssd_ctx *ctx, int32_t worker, const float **weights,
+                              int32_t *view);
+
+/* Counters: iterations done (Algorithm 1's num) and GLU calls done per worker
+ * (Algorithm 2's loc_update); stage and flags of the NEXT iteration.  Outputs
+ * may be NULL.  ssd_set_counters restores them (resume from a checkpoint whose
+ * buffers the caller has restored); loc_update must equal max(0, iter - W) when
+ * delay_k > 0 and 0 otherwise, else SSD_ERR_STATE. */
+ssd_status ssd_get_counters(const ssd_ctx *ctx, int64_t *iter, int64_t *loc_update,
+                            int32_t *next_stage, int32_t *next_flags);
+ssd_status ssd_set_counters(ssd_ctx *ctx, int64_t iter, int64_t loc_update);
+
+/* Changes the learning rates between iterations and re-derives c.  NaN keeps a
+ * value.  (The geometric-series argument behind grad_sync assumes a constant lr;
+ * after a change grad_sync is an estimate under the new lr.) */
+ssd_status ssd_set_lr(ssd_ctx *ctx, float lr, float lr_local);
+
+/* Resolved hyper-parameters as the kernels use them, and the derived c. */
+ssd_status ssd_get_hparams(const ssd_ctx *ctx, ssd_hparams *resolved, float *sync_scale);
+
+/* Launch shape of the streaming kernels: threads per block (multiple of 32,
+ * 64..1024) and resident blocks per SM (1..32).  0 keeps the default. */
+ssd_status ssd_set_launch(ssd_ctx *ctx, int32_t threads_per_block, int32_t blocks_per_sm);
+
+/* Number of kernels this context has launched so far. */
+int64_t ssd_kernel_launches(const ssd_ctx *ctx);
+
+/* Text for a status code (static storage). */
+const char *ssd_status_str(ssd_status status);
+
+/* Text of the last CUDA runtime error a call on this context returned as
+ * SSD_ERR_CUDA (static or context storage; empty string if none). */
+const char *ssd_last_cuda_error(const ssd_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SSD_SGD_H */

@@ -1,0 +1,506 @@
+// Host side of the SSD-SGD update library: context, argument validation, the
+// schedule state machine of Algorithm 1 / Algorithm 2, and the kernel launches.
+// The contract of every entry point is stated in include/ssd_sgd.h.
+#include "ssd_sgd.h"
+#include "ssd_kernels.cuh"
+
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+namespace {
+
+using namespace ssd;
+
+constexpr int64_t kMaxArena = int64_t(1) << 40;
+
+struct Device {
+    bool ready = false;
+    int id = -1;
+    int sms = 0;
+};
+
+}  // namespace
+
+struct ssd_ctx {
+    std::vector<int64_t> offsets;     // element offset of each tensor
+    int64_t n = 0;                    // arena length in elements
+    ssd_hparams hp{};                 // resolved
+    Scalars s{};
+    float *w = nullptr, *mom = nullptr;
+    float *w_loc[kMaxWorkers]{}, *pre[kMaxWorkers]{}, *w_dev[kMaxWorkers]{};
+    int64_t iter = 0, loc_update = 0;
+    int threads = 256, blocks_per_sm = 0;   // 0: as many as fit (occupancy query)
+    int64_t launches = 0;
+    Device dev;
+    std::string cuda_error;
+};
+
+namespace {
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+float derive_sync_scale(float lr, float m, int32_t k)
+{
+    if (k <= 0) return 0.0f;
+    return static_cast<float>((1.0 - static_cast<double>(m)) /
+                              (static_cast<double>(lr) * static_cast<double>(k)));
+}
+
+ssd_status padded_total(const ssd_layout *layout, int64_t *total, std::vector<int64_t> *offsets)
+{
+    if (!layout || !layout->numel) return SSD_ERR_ARG;
+    if (layout->num_tensors < 1) return SSD_ERR_LAYOUT;
+    int64_t pos = 0;
+    for (int32_t t = 0; t < layout->num_tensors; ++t) {
+        const int64_t c = layout->numel[t];
+        if (c < 0 || c >= kMaxArena) return SSD_ERR_LAYOUT;
+        if (offsets) offsets->push_back(pos);
+        pos += (c + 3) / 4 * 4;
+        if (pos >= kMaxArena) return SSD_ERR_LAYOUT;
+    }
+    if (pos == 0) return SSD_ERR_LAYOUT;
+    *total = pos;
+    return SSD_OK;
+}
+
+void schedule_of(const ssd_ctx *c, int64_t n, int32_t *stage, int32_t *flags)
+{
+    const int64_t W = c->hp.warmup_iters, k = c->hp.delay_k;
+    if (k == 0 || n < W) {
+        *stage = SSD_STAGE_WARMUP;
+        *flags = (k != 0 && n == W - 1) ? SSD_FLAG_COPY : 0;
+        return;
+    }
+    const int64_t d = n - W;
+    int32_t f = 0;
+    if (d == 0) f |= SSD_FLAG_FIRST;
+    if (d > 0 && d % k == 0) f |= SSD_FLAG_REFRESH;
+    if (d % k == k - 1) f |= SSD_FLAG_PULL;
+    *stage = SSD_STAGE_DELAY;
+    *flags = f;
+}
+
+ssd_status cuda_fail(ssd_ctx *c, cudaError_t e)
+{
+    c->cuda_error = cudaGetErrorString(e);
+    return SSD_ERR_CUDA;
+}
+
+ssd_status ensure_device(ssd_ctx *c)
+{
+    if (c->dev.ready) return SSD_OK;
+    int id = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&id);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, id);
+    if (e != cudaSuccess) {
+        (void)cudaGetLastError();
+        return cuda_fail(c, e);
+    }
+    c->dev.id = id;
+    c->dev.sms = sms;
+    c->dev.ready = true;
+    return SSD_OK;
+}
+
+// Grid for a sweep over n elements: one 128-bit vector per thread per trip, at most
+// `blocks_per_sm` resident blocks per SM so that the grid is one full wave.
+template <typename Kernel>
+ssd_status grid_for(ssd_ctx *c, Kernel kernel, int64_t n, int *grid)
+{
+    int per_sm = c->blocks_per_sm;
+    if (per_sm == 0) {
+        cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, c->threads, 0);
+        if (e != cudaSuccess) return cuda_fail(c, e);
+        if (per_sm < 1) per_sm = 1;
+    }
+    const int64_t nvec = n >> 2;
+    int64_t need = (nvec + c->threads - 1) / c->threads;
+    if (need < 1) need = 1;
+    const int64_t wave = static_cast<int64_t>(c->dev.sms) * per_sm;
+    *grid = static_cast<int>(need < wave ? need : wave);
+    return SSD_OK;
+}
+
+template <typename Kernel, typename Params>
+ssd_status launch(ssd_ctx *c, Kernel kernel, const Params &p, int64_t n, cudaStream_t stream)
+{
+    ssd_status st = ensure_device(c);
+    if (st != SSD_OK) return st;
+    int grid = 1;
+    st = grid_for(c, kernel, n, &grid);
+    if (st != SSD_OK) return st;
+    kernel<<<grid, c->threads, 0, stream>>>(p);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    c->launches += 1;
+    return SSD_OK;
+}
+
+constexpr int kSyncBatch = 8;   // gradient loads in flight per thread in sync_kernel
+constexpr int kStepBatch = 4;   // workers (3 loads each) in flight per thread in step_kernel
+
+ssd_status check_grads(const ssd_ctx *c, const void *const *grads)
+{
+    if (!grads) return SSD_ERR_ARG;
+    for (int i = 0; i < c->hp.K; ++i) {
+        if (!grads[i]) return SSD_ERR_ARG;
+        if (!aligned16(grads[i])) return SSD_ERR_ALIGN;
+    }
+    return SSD_OK;
+}
+
+ssd_status launch_sync(ssd_ctx *c, const void *const *grads, int flags, cudaStream_t stream)
+{
+    SyncParams p{};
+    for (int i = 0; i < c->hp.K; ++i) {
+        p.g[i] = grads[i];
+        p.w_loc[i] = c->w_loc[i];
+    }
+    p.w = c->w;
+    p.mom = c->mom;
+    p.n = c->n;
+    p.K = c->hp.K;
+    p.flags = flags;
+    p.s = c->s;
+    if (c->hp.grad_dtype == SSD_BF16)
+        return launch(c, sync_kernel<kBF16, kSyncBatch>, p, c->n, stream);
+    return launch(c, sync_kernel<kF32, kSyncBatch>, p, c->n, stream);
+}
+
+ssd_status launch_glu(ssd_ctx *c, int worker, const void *grad, int flags, cudaStream_t stream)
+{
+    GluParams p{};
+    p.g = grad;
+    p.w_loc = c->w_loc[worker];
+    p.pre = c->pre[worker];
+    p.w_dev = c->w_dev[worker];
+    p.w = c->w;
+    p.n = c->n;
+    p.flags = flags;
+    p.s = c->s;
+    if (c->hp.grad_dtype == SSD_BF16) return launch(c, glu_kernel<kBF16>, p, c->n, stream);
+    return launch(c, glu_kernel<kF32>, p, c->n, stream);
+}
+
+ssd_status launch_step(ssd_ctx *c, const void *const *grads, int flags, cudaStream_t stream)
+{
+    StepParams p{};
+    for (int i = 0; i < c->hp.K; ++i) {
+        p.g[i] = grads[i];
+        p.w_loc[i] = c->w_loc[i];
+        p.pre[i] = c->pre[i];
+        p.w_dev[i] = c->w_dev[i];
+    }
+    p.w = c->w;
+    p.mom = c->mom;
+    p.n = c->n;
+    p.K = c->hp.K;
+    p.flags = flags;
+    p.s = c->s;
+    if (c->hp.grad_dtype == SSD_BF16)
+        return launch(c, step_kernel<kBF16, kStepBatch>, p, c->n, stream);
+    return launch(c, step_kernel<kF32, kStepBatch>, p, c->n, stream);
+}
+
+ssd_status launch_copy(ssd_ctx *c, int first_worker, int count, cudaStream_t stream)
+{
+    CopyParams p{};
+    for (int i = 0; i < count; ++i) p.dst[i] = c->w_loc[first_worker + i];
+    p.src = c->w;
+    p.n = c->n;
+    p.K = count;
+    return launch(c, copy_kernel, p, c->n, stream);
+}
+
+void advance(ssd_ctx *c)
+{
+    int32_t stage, flags;
+    schedule_of(c, c->iter, &stage, &flags);
+    c->iter += 1;
+    if (stage == SSD_STAGE_DELAY) c->loc_update += 1;
+}
+
+}  // namespace
+
+extern "C" {
+
+ssd_status ssd_arena_numel(const ssd_layout *layout, int64_t *padded_numel)
+{
+    if (!padded_numel) return SSD_ERR_ARG;
+    return padded_total(layout, padded_numel, nullptr);
+}
+
+ssd_status ssd_init(ssd_ctx **out, const ssd_layout *layout, const ssd_hparams *hp,
+                    const ssd_buffers *b)
+{
+    if (!out) return SSD_ERR_ARG;
+    *out = nullptr;
+    if (!layout || !hp || !b) return SSD_ERR_ARG;
+    if (hp->K < 1 || hp->K > SSD_MAX_WORKERS) return SSD_ERR_ARG;
+    if (!(hp->lr > 0.0f) || !std::isfinite(hp->lr)) return SSD_ERR_ARG;
+    if (!(hp->momentum >= 0.0f && hp->momentum < 1.0f)) return SSD_ERR_ARG;
+    if (!std::isfinite(hp->wd)) return SSD_ERR_ARG;
+    if (hp->warmup_iters < 0 || hp->delay_k < 0) return SSD_ERR_ARG;
+    if (hp->grad_dtype != SSD_F32 && hp->grad_dtype != SSD_BF16) return SSD_ERR_ARG;
+    if (std::isinf(hp->lr_local) || std::isinf(hp->alpha) || std::isinf(hp->beta) ||
+        std::isinf(hp->rescale))
+        return SSD_ERR_ARG;
+    if (!b->w || !b->mom || !b->w_loc || !b->pre || !b->w_dev) return SSD_ERR_ARG;
+
+    ssd_ctx *c = new (std::nothrow) ssd_ctx;
+    if (!c) return SSD_ERR_NOMEM;
+    ssd_status st = padded_total(layout, &c->n, &c->offsets);
+    if (st != SSD_OK) {
+        delete c;
+        return st;
+    }
+    std::vector<const void *> all{b->w, b->mom};
+    for (int i = 0; i < hp->K; ++i) {
+        all.push_back(b->w_loc[i]);
+        all.push_back(b->pre[i]);
+        all.push_back(b->w_dev[i]);
+    }
+    for (const void *p : all) {
+        if (!p) st = SSD_ERR_ARG;
+        else if (!aligned16(p) && st == SSD_OK) st = SSD_ERR_ALIGN;
+    }
+    // No two state buffers may share an address: every element is read and written
+    // by one thread only, which holds only if the buffers are distinct.
+    for (size_t x = 0; x < all.size() && st == SSD_OK; ++x)
+        for (size_t y = x + 1; y < all.size(); ++y)
+            if (all[x] == all[y]) st = SSD_ERR_ARG;
+    if (st != SSD_OK) {
+        delete c;
+        return st;
+    }
+
+    c->hp = *hp;
+    if (std::isnan(hp->lr_local)) c->hp.lr_local = 4.0f * hp->lr;
+    if (std::isnan(hp->alpha)) c->hp.alpha = 2.0f;
+    if (std::isnan(hp->beta)) c->hp.beta = 0.5f;
+    if (std::isnan(hp->rescale)) c->hp.rescale = static_cast<float>(1.0 / static_cast<double>(hp->K));
+    c->s.lr = c->hp.lr;
+    c->s.m = c->hp.momentum;
+    c->s.wd = c->hp.wd;
+    c->s.rescale = c->hp.rescale;
+    c->s.lr_loc = c->hp.lr_local;
+    c->s.alpha = c->hp.alpha;
+    c->s.beta = c->hp.beta;
+    c->s.c = derive_sync_scale(c->hp.lr, c->hp.momentum, c->hp.delay_k);
+    c->w = b->w;
+    c->mom = b->mom;
+    for (int i = 0; i < hp->K; ++i) {
+        c->w_loc[i] = b->w_loc[i];
+        c->pre[i] = b->pre[i];
+        c->w_dev[i] = b->w_dev[i];
+    }
+    *out = c;
+    return SSD_OK;
+}
+
+void ssd_destroy(ssd_ctx *ctx) { delete ctx; }
+
+ssd_status ssd_tensor_offset(const ssd_ctx *ctx, int32_t tensor, int64_t *elem_offset)
+{
+    if (!ctx || !elem_offset) return SSD_ERR_ARG;
+    if (tensor < 0 || tensor >= static_cast<int32_t>(ctx->offsets.size())) return SSD_ERR_ARG;
+    *elem_offset = ctx->offsets[tensor];
+    return SSD_OK;
+}
+
+ssd_status ssd_schedule(const ssd_ctx *ctx, int64_t iter, int32_t *stage, int32_t *flags)
+{
+    if (!ctx || !stage || !flags || iter < 0) return SSD_ERR_ARG;
+    schedule_of(ctx, iter, stage, flags);
+    return SSD_OK;
+}
+
+ssd_status ssd_server_sync_update(ssd_ctx *ctx, const void *const *grads, void *cuda_stream)
+{
+    if (!ctx) return SSD_ERR_ARG;
+    ssd_status st = check_grads(ctx, grads);
+    if (st != SSD_OK) return st;
+    return launch_sync(ctx, grads, 0, static_cast<cudaStream_t>(cuda_stream));
+}
+
+ssd_status ssd_worker_glu_update(ssd_ctx *ctx, int32_t worker, const void *grad, int32_t flags,
+                                 void *cuda_stream)
+{
+    if (!ctx || !grad) return SSD_ERR_ARG;
+    if (worker < 0 || worker >= ctx->hp.K) return SSD_ERR_ARG;
+    if (flags & ~(SSD_FLAG_FIRST | SSD_FLAG_REFRESH | SSD_FLAG_PULL)) return SSD_ERR_ARG;
+    if (ctx->hp.delay_k == 0) return SSD_ERR_STATE;
+    if (!aligned16(grad)) return SSD_ERR_ALIGN;
+    return launch_glu(ctx, worker, grad, flags, static_cast<cudaStream_t>(cuda_stream));
+}
+
+ssd_status ssd_worker_local_step(ssd_ctx *ctx, int32_t worker, const void *grad, void *cuda_stream)
+{
+    if (!ctx) return SSD_ERR_ARG;
+    if (worker < 0 || worker >= ctx->hp.K) return SSD_ERR_ARG;
+    int32_t stage, flags;
+    schedule_of(ctx, ctx->iter, &stage, &flags);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (stage == SSD_STAGE_WARMUP) {
+        if (flags & SSD_FLAG_COPY) return launch_copy(ctx, worker, 1, stream);
+        return SSD_OK;
+    }
+    if (!grad) return SSD_ERR_ARG;
+    if (!aligned16(grad)) return SSD_ERR_ALIGN;
+    return launch_glu(ctx, worker, grad, flags, stream);
+}
+
+ssd_status ssd_advance(ssd_ctx *ctx)
+{
+    if (!ctx) return SSD_ERR_ARG;
+    advance(ctx);
+    return SSD_OK;
+}
+
+ssd_status ssd_step(ssd_ctx *ctx, const void *const *grads, void *cuda_stream)
+{
+    if (!ctx) return SSD_ERR_ARG;
+    ssd_status st = check_grads(ctx, grads);
+    if (st != SSD_OK) return st;
+    int32_t stage, flags;
+    schedule_of(ctx, ctx->iter, &stage, &flags);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    st = (stage == SSD_STAGE_WARMUP) ? launch_sync(ctx, grads, flags & SSD_FLAG_COPY, stream)
+                                     : launch_step(ctx, grads, flags, stream);
+    if (st != SSD_OK) return st;
+    advance(ctx);
+    return SSD_OK;
+}
+
+ssd_status ssd_step_host(ssd_ctx *ctx, const void *const *host_grads, void *const *staging,
+                         float *host_w_out, void *cuda_stream)
+{
+    if (!ctx || !host_grads || !staging) return SSD_ERR_ARG;
+    for (int i = 0; i < ctx->hp.K; ++i) {
+        if (!host_grads[i] || !staging[i]) return SSD_ERR_ARG;
+        if (!aligned16(staging[i])) return SSD_ERR_ALIGN;
+    }
+    ssd_status st = ensure_device(ctx);
+    if (st != SSD_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const size_t gbytes = static_cast<size_t>(ctx->n) * (ctx->hp.grad_dtype == SSD_BF16 ? 2 : 4);
+    for (int i = 0; i < ctx->hp.K; ++i) {
+        cudaError_t e = cudaMemcpyAsync(staging[i], host_grads[i], gbytes, cudaMemcpyHostToDevice, stream);
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+    }
+    st = ssd_step(ctx, const_cast<const void *const *>(staging), cuda_stream);
+    if (st != SSD_OK) return st;
+    if (host_w_out) {
+        cudaError_t e = cudaMemcpyAsync(host_w_out, ctx->w, static_cast<size_t>(ctx->n) * 4,
+                                        cudaMemcpyDeviceToHost, stream);
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+    }
+    return SSD_OK;
+}
+
+ssd_status ssd_broadcast_weights(ssd_ctx *ctx, void *cuda_stream)
+{
+    if (!ctx) return SSD_ERR_ARG;
+    return launch_copy(ctx, 0, ctx->hp.K, static_cast<cudaStream_t>(cuda_stream));
+}
+
+ssd_status ssd_worker_weights(const ssd_ctx *ctx, int32_t worker, const float **weights, int32_t *view)
+{
+    if (!ctx) return SSD_ERR_ARG;
+    if (worker < 0 || worker >= ctx->hp.K) return SSD_ERR_ARG;
+    int32_t v = SSD_VIEW_GLOBAL;
+    if (ctx->iter > 0) {
+        int32_t stage, flags;
+        schedule_of(ctx, ctx->iter - 1, &stage, &flags);
+        if (stage == SSD_STAGE_WARMUP) v = (flags & SSD_FLAG_COPY) ? SSD_VIEW_LOCAL : SSD_VIEW_GLOBAL;
+        else v = (flags & SSD_FLAG_PULL) ? SSD_VIEW_DEVICE : SSD_VIEW_LOCAL;
+    }
+    if (view) *view = v;
+    if (weights)
+        *weights = v == SSD_VIEW_GLOBAL ? ctx->w : v == SSD_VIEW_LOCAL ? ctx->w_loc[worker] : ctx->w_dev[worker];
+    return SSD_OK;
+}
+
+ssd_status ssd_get_counters(const ssd_ctx *ctx, int64_t *iter, int64_t *loc_update,
+                            int32_t *next_stage, int32_t *next_flags)
+{
+    if (!ctx) return SSD_ERR_ARG;
+    int32_t stage, flags;
+    schedule_of(ctx, ctx->iter, &stage, &flags);
+    if (iter) *iter = ctx->iter;
+    if (loc_update) *loc_update = ctx->loc_update;
+    if (next_stage) *next_stage = stage;
+    if (next_flags) *next_flags = flags;
+    return SSD_OK;
+}
+
+ssd_status ssd_set_counters(ssd_ctx *ctx, int64_t iter, int64_t loc_update)
+{
+    if (!ctx || iter < 0 || loc_update < 0) return SSD_ERR_ARG;
+    int64_t expect = 0;
+    if (ctx->hp.delay_k > 0 && iter > ctx->hp.warmup_iters) expect = iter - ctx->hp.warmup_iters;
+    if (loc_update != expect) return SSD_ERR_STATE;
+    ctx->iter = iter;
+    ctx->loc_update = loc_update;
+    return SSD_OK;
+}
+
+ssd_status ssd_set_lr(ssd_ctx *ctx, float lr, float lr_local)
+{
+    if (!ctx) return SSD_ERR_ARG;
+    if (!std::isnan(lr) && (!(lr > 0.0f) || !std::isfinite(lr))) return SSD_ERR_ARG;
+    if (std::isinf(lr_local)) return SSD_ERR_ARG;
+    if (!std::isnan(lr)) {
+        ctx->hp.lr = lr;
+        ctx->s.lr = lr;
+        ctx->s.c = derive_sync_scale(lr, ctx->hp.momentum, ctx->hp.delay_k);
+    }
+    if (!std::isnan(lr_local)) {
+        ctx->hp.lr_local = lr_local;
+        ctx->s.lr_loc = lr_local;
+    }
+    return SSD_OK;
+}
+
+ssd_status ssd_get_hparams(const ssd_ctx *ctx, ssd_hparams *resolved, float *sync_scale)
+{
+    if (!ctx) return SSD_ERR_ARG;
+    if (resolved) *resolved = ctx->hp;
+    if (sync_scale) *sync_scale = ctx->s.c;
+    return SSD_OK;
+}
+
+ssd_status ssd_set_launch(ssd_ctx *ctx, int32_t threads_per_block, int32_t blocks_per_sm)
+{
+    if (!ctx) return SSD_ERR_ARG;
+    if (threads_per_block != 0 &&
+        (threads_per_block < 64 || threads_per_block > kMaxThreads || threads_per_block % 32 != 0))
+        return SSD_ERR_ARG;
+    if (blocks_per_sm < 0 || blocks_per_sm > 32) return SSD_ERR_ARG;
+    if (threads_per_block) ctx->threads = threads_per_block;
+    ctx->blocks_per_sm = blocks_per_sm;
+    return SSD_OK;
+}
+
+int64_t ssd_kernel_launches(const ssd_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+const char *ssd_status_str(ssd_status status)
+{
+    switch (status) {
+    case SSD_OK: return "ok";
+    case SSD_ERR_ARG: return "invalid argument";
+    case SSD_ERR_ALIGN: return "device pointer not 16-byte aligned";
+    case SSD_ERR_LAYOUT: return "invalid parameter layout";
+    case SSD_ERR_STATE: return "call not valid in the current stage";
+    case SSD_ERR_CUDA: return "CUDA runtime error";
+    case SSD_ERR_NOMEM: return "out of host memory";
+    }
+    return "unknown status";
+}
+
+const char *ssd_last_cuda_error(const ssd_ctx *ctx) { return ctx ? ctx->cuda_error.c_str() : ""; }
+
+}  // extern "C"

@@ -1,0 +1,76 @@
+"""Helpers shared by the GPU parity tests: run a schedule on both sides and compare bit patterns."""
+import numpy as np
+import torch
+
+import oracle
+from paper_2012_05396_b200 import binding as B
+from paper_2012_05396_b200 import synth
+from paper_2012_05396_b200.state import DeviceState
+
+# The arithmetic is defined operation by operation (binary32, no fused multiply-add, fixed
+# summation order), so the CUDA result is unique and must equal the oracle's bit for bit.  That
+# is stricter than the stated floating-point bar, which is also asserted:
+REL_TOL, ABS_TOL = 1e-6, 1e-7
+
+
+def bits(a):
+    if isinstance(a, torch.Tensor):
+        a = a.detach().cpu().numpy()
+    return np.ascontiguousarray(a).view(np.uint32)
+
+
+def assert_same(got, want, what, idx=None):
+    g = got.detach().cpu().numpy() if isinstance(got, torch.Tensor) else got
+    if idx is not None:
+        g = g[idx]
+    gb, wb = bits(g), bits(want)
+    if not np.array_equal(gb, wb):
+        bad = np.nonzero(gb != wb)[0]
+        j = int(bad[0])
+        raise AssertionError(f"{what}: {bad.size} of {wb.size} elements differ; first at {j}: "
+                             f"cuda {g[j]!r} oracle {want[j]!r}")
+    finite = np.isfinite(want)
+    err = np.abs(g[finite].astype(np.float64) - want[finite].astype(np.float64))
+    assert np.all(err <= ABS_TOL + REL_TOL * np.abs(want[finite].astype(np.float64))), what
+
+
+def make_hp(K, lr, m, W, k, wd=0.0, lr_loc=None, alpha=2.0, beta=0.5, rescale=None, bf16=False):
+    """The same hyper-parameters for both sides (defaults resolved by each side on its own)."""
+    nan = float("nan")
+    o = oracle.Hyper(K=K, lr=lr, m=m, W=W, k=k, wd=wd, lr_loc=lr_loc, alpha=alpha, beta=beta,
+                     rescale=rescale, grad_bf16=bf16)
+    c = B.make_hparams(K, lr, m, W, k, wd=wd, lr_local=nan if lr_loc is None else lr_loc,
+                       alpha=alpha, beta=beta, rescale=nan if rescale is None else rescale,
+                       grad_dtype=B.SSD_BF16 if bf16 else B.SSD_F32)
+    return o, c
+
+
+def oracle_grad(g: torch.Tensor, bf16: bool):
+    """Device gradient tensor -> the numpy array the oracle consumes."""
+    if bf16:
+        return synth.bf16_bits(g)
+    return g.detach().cpu().numpy()
+
+
+def compare_states(dev: DeviceState, ref: oracle.State, tag, idx=None):
+    assert_same(dev.w, ref.w, f"{tag} w", idx)
+    assert_same(dev.mom, ref.mom, f"{tag} mom", idx)
+    for i in range(dev.K):
+        assert_same(dev.w_loc[i], ref.w_loc[i], f"{tag} w_loc[{i}]", idx)
+        assert_same(dev.pre[i], ref.pre[i], f"{tag} pre[{i}]", idx)
+        assert_same(dev.w_dev[i], ref.w_dev[i], f"{tag} w_dev[{i}]", idx)
+    it, lu, _, _ = dev.ctx.ssd_get_counters()
+    assert (it, lu) == (ref.iter, ref.loc_update), tag
+    for i in range(dev.K):
+        assert dev.ctx.ssd_worker_weights(i)[1] == ref.view, tag
+
+
+def gpu_iteration(dev: DeviceState, grads, mode):
+    """One iteration on the GPU: 'fused' = ssd_step, 'split' = server + K local steps + advance."""
+    if mode == "fused":
+        dev.ctx.ssd_step(grads)
+    else:
+        dev.ctx.ssd_server_sync_update(grads)
+        for i in range(dev.K):
+            dev.ctx.ssd_worker_local_step(i, grads[i])
+        dev.ctx.ssd_advance()

@@ -1,0 +1,219 @@
+"""CUDA path against the CPU oracle, element by element, through the C ABI (needs a B200)."""
+import itertools
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2012_05396_b200 import binding as B
+from paper_2012_05396_b200 import synth
+from paper_2012_05396_b200.state import DeviceState
+from tests import golden_trace
+from tests.gpu_common import (assert_same, compare_states, gpu_iteration, make_hp, oracle_grad)
+
+pytestmark = pytest.mark.gpu
+f32 = np.float32
+
+
+@pytest.mark.parametrize("mode", ["fused", "split"])
+@pytest.mark.parametrize("name", golden_trace.ALL)
+def test_hand_traces_on_the_gpu(name, mode):
+    tr = golden_trace.load(name)
+    h = tr.hp
+    K = int(h["K"])
+    _, hp = make_hp(K, h["lr"], h["m"], int(h["W"]), int(h["k"]), wd=h["wd"], lr_loc=h["lr_loc"],
+                    alpha=h["alpha"], beta=h["beta"], rescale=h["rescale"])
+    dev = DeviceState([len(tr.w0)], hp, torch.from_numpy(tr.w0))
+    for it in tr.iters:
+        stage, flags = dev.ctx.ssd_schedule(it.n)
+        assert (stage, flags) == (it.stage, it.flags)
+        grads = [torch.from_numpy(it.grads[i]).cuda() for i in range(K)]
+        gpu_iteration(dev, grads, mode)
+        torch.cuda.synchronize()
+        assert dev.ctx.ssd_worker_weights(0)[1] == it.view
+        for key, exp in it.server.items():
+            assert_same(getattr(dev, key), exp, f"{name} iter {it.n} {key}")
+        for (key, i), exp in it.worker.items():
+            assert_same(getattr(dev, key)[i], exp, f"{name} iter {it.n} {key}[{i}]")
+
+
+def run_both(numels, K, W, k, iters, sigma, mode, wd=0.0, bf16=False, seed=synth.SEED, lr=0.1, m=0.9,
+             check_every=1, w0=None):
+    ohp, chp = make_hp(K, lr, m, W, k, wd=wd, bf16=bf16)
+    lay = synth.Layout("t")
+    for n in numels:
+        lay.add("x", n, "he", 16)
+    if w0 is None:
+        w0 = synth.init_weights(lay, seed)
+    dev = DeviceState(lay.numels, chp, w0)
+    ref = oracle.State(ohp, w0.numpy())
+    mask = synth.valid_mask(lay, "cuda")
+    for n in range(iters):
+        grads = [synth.gradient(lay, n, i, sigma, seed, "cuda", mask) for i in range(K)]
+        if bf16:
+            grads = [synth.to_bf16(g) for g in grads]
+        gpu_iteration(dev, grads, mode)
+        stage, flags = ref.step([oracle_grad(g, bf16) for g in grads])
+        if (n + 1) % check_every == 0 or n == iters - 1:
+            torch.cuda.synchronize()
+            compare_states(dev, ref, f"iter {n} stage {stage} flags {flags}")
+    return dev, ref
+
+
+@pytest.mark.parametrize("mode", ["fused", "split"])
+@pytest.mark.parametrize("bf16", [False, True])
+def test_tiny_and_ragged_sizes(mode, bf16):
+    # vector tails (n % 4 != 0), single elements, several tensors with padding between them
+    for numels, K, W, k in [([1], 1, 1, 1), ([3], 2, 0, 2), ([5], 3, 2, 3), ([7, 1, 2], 5, 1, 2),
+                            ([17], 4, 2, 4), ([4, 4], 8, 3, 1), ([1023], 17, 2, 2), ([4097, 33], 32, 1, 3)]:
+        run_both(numels, K, W, k, W + 3 * max(k, 1) + 2, 0.05, mode, wd=0.01, bf16=bf16)
+
+
+@pytest.mark.parametrize("mode", ["fused", "split"])
+def test_every_small_schedule(mode):
+    for W, k in itertools.product(range(4), range(4)):
+        run_both([37, 6], 3, W, k, 11, 0.1, mode, wd=0.001)
+
+
+def test_multi_wave_grid_with_partial_last_trip():
+    # more vectors than one wave of blocks covers, the last trip only partly filled, smallest launch shape
+    ohp, chp = make_hp(6, 0.1, 0.9, 1, 2)
+    n = 148 * 64 * 4 * 5 + 36
+    lay = synth.flat(n)
+    w0 = synth.init_weights(lay)
+    dev = DeviceState(lay.numels, chp, w0)
+    dev.ctx.ssd_set_launch(64, 1)
+    ref = oracle.State(ohp, w0.numpy())
+    for it in range(5):
+        grads = [synth.gradient(lay, it, i, 0.02, device="cuda") for i in range(6)]
+        gpu_iteration(dev, grads, "fused")
+        ref.step([oracle_grad(g, False) for g in grads])
+    torch.cuda.synchronize()
+    compare_states(dev, ref, "multi-wave")
+
+
+def test_config_resnet20_K4():
+    # ResNet-20 layout, K=4, He-init, N(0, 1e-2) gradients, lr 0.1, m 0.9, W=2, k=4, 20 iterations
+    lay = synth.get_layout("resnet20")
+    for mode in ("fused", "split"):
+        run_both(lay.numels, 4, 2, 4, 20, 1e-2, mode)
+
+
+def test_config_resnet56_K8():
+    # ResNet-56 layout, K=8, W=5, k=4, 100 iterations
+    lay = synth.get_layout("resnet56")
+    run_both(lay.numels, 8, 5, 4, 100, 1e-2, "fused", check_every=7)
+
+
+def test_server_alone_is_synchronous_sgd():
+    # zero delay: ssd_step never leaves the warm-up stage and equals ssd_server_sync_update alone
+    lay = synth.get_layout("resnet20")
+    ohp, chp = make_hp(4, 0.1, 0.9, 3, 0, wd=1e-4)
+    w0 = synth.init_weights(lay)
+    a, b = DeviceState(lay.numels, chp, w0), DeviceState(lay.numels, chp, w0)
+    ref = oracle.State(ohp, w0.numpy())
+    for n in range(6):
+        grads = [synth.gradient(lay, n, i, 1e-2, device="cuda") for i in range(4)]
+        a.ctx.ssd_step(grads)
+        b.ctx.ssd_server_sync_update(grads)
+        ref.step([oracle_grad(g, False) for g in grads])
+    torch.cuda.synchronize()
+    compare_states(a, ref, "k=0")
+    assert_same(b.w, ref.w, "server-only w")
+    assert_same(b.mom, ref.mom, "server-only mom")
+    assert b.ctx.ssd_get_counters()[0] == 0
+
+
+def test_glu_update_flags_one_by_one():
+    # ssd_worker_glu_update with explicit flags from primed uniform(-1,1) state (sweep workload)
+    n = (1 << 16) + 8
+    for bf16 in (False, True):
+        ohp, chp = make_hp(2, 0.1, 0.9, 0, 4, wd=0.01, bf16=bf16)
+        for flags in range(8):
+            w0 = synth.uniform_buffer(synth.STREAM_WEIGHT, n)
+            dev = DeviceState([n], chp, w0)
+            ref = oracle.State(ohp, w0.numpy())
+            for i in range(2):
+                wl = synth.uniform_buffer(synth.STREAM_WLOC, n, worker=i)
+                pr = synth.uniform_buffer(synth.STREAM_PRE, n, worker=i)
+                dev.w_loc[i].copy_(wl); dev.pre[i].copy_(pr)
+                ref.w_loc[i][:] = wl.numpy(); ref.pre[i][:] = pr.numpy()
+                g = synth.uniform_buffer(synth.STREAM_GRAD, n, worker=i, device="cuda")
+                if bf16:
+                    g = synth.to_bf16(g)
+                dev.ctx.ssd_worker_glu_update(i, g, flags)
+                oracle.glu_update(ohp, oracle_grad(g, bf16), ref.w_loc[i], ref.pre[i], ref.w_dev[i],
+                                  ref.w, flags)
+            torch.cuda.synchronize()
+            for i in range(2):
+                for name in ("w_loc", "pre", "w_dev"):
+                    assert_same(getattr(dev, name)[i], getattr(ref, name)[i], f"flags {flags} {name}[{i}]")
+            assert_same(dev.w, ref.w, "w untouched")
+
+
+def test_broadcast_weights_and_zero_warmup():
+    lay = synth.get_layout("resnet20")
+    ohp, chp = make_hp(3, 0.1, 0.9, 0, 2)
+    w0 = synth.init_weights(lay)
+    dev = DeviceState(lay.numels, chp, w0)
+    for t in dev.w_loc:
+        t.fill_(float("nan"))
+    dev.ctx.ssd_broadcast_weights()
+    torch.cuda.synchronize()
+    for t in dev.w_loc:
+        assert torch.equal(t, dev.w)
+    ref = oracle.State(ohp, w0.numpy())
+    for n in range(5):
+        grads = [synth.gradient(lay, n, i, 1e-2, device="cuda") for i in range(3)]
+        dev.ctx.ssd_step(grads)
+        ref.step([oracle_grad(g, False) for g in grads])
+    torch.cuda.synchronize()
+    compare_states(dev, ref, "W=0")
+
+
+def test_checkpoint_resume_is_bit_exact():
+    lay = synth.get_layout("resnet20")
+    _, chp = make_hp(4, 0.1, 0.9, 2, 4)
+    w0 = synth.init_weights(lay)
+    full = DeviceState(lay.numels, chp, w0)
+    half = DeviceState(lay.numels, chp, w0)
+    def grads(n):
+        return [synth.gradient(lay, n, i, 1e-2, device="cuda") for i in range(4)]
+    for n in range(14):
+        full.ctx.ssd_step(grads(n))
+    for n in range(7):
+        half.ctx.ssd_step(grads(n))
+    it, lu, _, _ = half.ctx.ssd_get_counters()
+    resumed = DeviceState(lay.numels, chp, half.w)          # a new context over restored buffers
+    resumed.mom.copy_(half.mom)
+    for i in range(4):
+        resumed.w_loc[i].copy_(half.w_loc[i]); resumed.pre[i].copy_(half.pre[i])
+        resumed.w_dev[i].copy_(half.w_dev[i])
+    resumed.ctx.ssd_set_counters(it, lu)
+    for n in range(7, 14):
+        resumed.ctx.ssd_step(grads(n))
+    torch.cuda.synchronize()
+    for name in ("w", "mom"):
+        assert_same(getattr(resumed, name), getattr(full, name).cpu().numpy(), name)
+    for i in range(4):
+        for name in ("w_loc", "pre", "w_dev"):
+            assert_same(getattr(resumed, name)[i], getattr(full, name)[i].cpu().numpy(), f"{name}[{i}]")
+
+
+def test_step_host_moves_gradients_and_returns_weights():
+    lay = synth.get_layout("resnet20")
+    ohp, chp = make_hp(4, 0.1, 0.9, 1, 2)
+    w0 = synth.init_weights(lay)
+    dev = DeviceState(lay.numels, chp, w0)
+    ref = oracle.State(ohp, w0.numpy())
+    staging = [torch.empty(dev.n, dtype=torch.float32, device="cuda") for _ in range(4)]
+    w_out = torch.empty(dev.n, dtype=torch.float32).pin_memory()
+    for n in range(4):
+        host = [synth.gradient(lay, n, i, 1e-2).pin_memory() for i in range(4)]
+        dev.ctx.ssd_step_host(host, staging, w_out)
+        torch.cuda.synchronize()
+        ref.step([h.numpy() for h in host])
+        assert_same(w_out, ref.w, f"host w iter {n}")
+    compare_states(dev, ref, "step_host")
+    assert dev.ctx.ssd_kernel_launches() == 4
