@@ -1,0 +1,375 @@
+#!/usr/bin/env python
+"""Benchmark of the SSD-SGD update path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+One "step" is one whole iteration of the method (server aggregate + momentum-SGD and all K
+workers' GLU updates, with the pre_weight refreshes and pulls the schedule asks for) over one
+batch of synthetic gradients, through the fused ssd_step entry point.  The timed steps are all
+in the steps-delay stage (the SSD-SGD warm-up stage and the first GLU call run before timing).
+Prints ONE JSON line.  With --gpus N > 1 (under torchrun) every rank runs an independent
+replica: the method's state lives on one GPU and there is no exchange between GPUs.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+METRIC = "ssd_sgd_update_bandwidth"
+UNIT = "GB/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+# name -> layout, workers, server lr, momentum, SSD warm-up iterations, delay steps, gradient sigma
+WORKLOADS = {
+    "resnet20_K4": dict(layout="resnet20", K=4, lr=0.1, m=0.9, W=2, k=4, sigma=1e-2),
+    "resnet56_K8": dict(layout="resnet56", K=8, lr=0.1, m=0.9, W=5, k=4, sigma=1e-2),
+    "resnet50_K8": dict(layout="resnet50", K=8, lr=0.1, m=0.9, W=8, k=4, sigma=1e-3),
+    "vgg16_K16": dict(layout="vgg16", K=16, lr=0.01, m=0.9, W=4, k=4, sigma=1e-3),
+}
+DEFAULT_WORKLOAD = "vgg16_K16"
+
+# DRAM bytes per launch of step_kernel from an ncu capture (dram__bytes_read.sum +
+# dram__bytes_write.sum), valid only for the kernel sources with this digest.
+NCU_TRAFFIC = {"digest": None, "workload": None, "bytes_per_launch": None}
+
+
+def kernel_digest() -> str:
+    h = hashlib.sha256()
+    for name in ("ssd_kernels.cuh", "ssd_sgd.cu"):
+        with open(os.path.join(ROOT, "paper_2012_05396_b200", "csrc", name), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def step_bytes_per_param(K: int, sg: int, flags: int) -> int:
+    """Algorithmic bytes one fused delay-stage step moves per parameter: K gradients, K local
+    weights read and written, K pre_weights read, w and mom read and written; a refresh adds K
+    pre_weight stores, a pull adds K device-weight stores (and trades nothing else)."""
+    b = K * (sg + 12) + 16
+    if flags & 2:       # refresh
+        b += 4 * K
+    if flags & 4:       # pull
+        b += 4 * K
+    return b
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock samples of one GPU while the timed region runs."""
+
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.file = None
+
+    def start(self):
+        try:
+            self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.QUERY}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=self.file, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        sm, smax, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.file.read().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                smax.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.file.close()
+        os.unlink(self.file.name)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), reasons=sorted(reasons),
+                       samples=len(sm))
+        return out
+
+
+def dist_setup(n_gpus: int):
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if n_gpus > 1 and world != n_gpus:
+        raise SystemExit(f"--gpus {n_gpus} needs torchrun with {n_gpus} ranks (WORLD_SIZE={world})")
+    return world, rank, local
+
+
+def oracle_sample_run(wl, n_sample: int, steps: int, grads_host, w0_host):
+    """Times the CPU oracle, as it stands, on the first n_sample arena elements for `steps`
+    delay-stage iterations.  Returns (seconds, bytes moved, params updated, threads used)."""
+    import oracle
+    hp = oracle.Hyper(K=wl["K"], lr=wl["lr"], m=wl["m"], W=wl["W"], k=wl["k"])
+    st = oracle.State(hp, w0_host[:n_sample], fill=0.0)
+    for n in range(wl["W"] + 1):                      # SSD warm-up stage and the first GLU call: untimed
+        st.step(grads_host[n % len(grads_host)])
+    moved = 0
+    t0 = time.perf_counter()
+    for n in range(steps):
+        _, flags = st.step(grads_host[n % len(grads_host)])
+        moved += step_bytes_per_param(wl["K"], 4, flags) * n_sample
+    dt = time.perf_counter() - t0
+    return dt, moved, n_sample * steps, 1
+
+
+def run_reference(args, wl_name, wl):
+    """--impl reference: the CPU oracle on the host cores, a bounded sample per step."""
+    from paper_2012_05396_b200 import synth
+    lay = synth.get_layout(wl["layout"])
+    n_sample = min(lay.padded_numel, 1 << 22)
+    K = wl["K"]
+    w0 = synth.init_weights(lay)[:n_sample].numpy() if lay.padded_numel <= (1 << 22) else \
+        synth.normal(synth.stream_key(synth.SEED, synth.STREAM_WEIGHT), n_sample, 0.02).numpy()
+    sets = []
+    for s in range(2):
+        sets.append([synth.normal(synth.stream_key(synth.SEED, synth.STREAM_GRAD, s, i), n_sample,
+                                  wl["sigma"]).numpy() for i in range(K)])
+    import oracle
+    hp = oracle.Hyper(K=K, lr=wl["lr"], m=wl["m"], W=wl["W"], k=wl["k"])
+    st = oracle.State(hp, w0, fill=0.0)
+    for n in range(wl["W"] + 1 + args.warmup):
+        st.step(sets[n % 2])
+    moved = 0
+    t0 = time.perf_counter()
+    for n in range(args.steps):
+        _, flags = st.step(sets[n % 2])
+        moved += step_bytes_per_param(K, 4, flags) * n_sample
+    dt = time.perf_counter() - t0
+    gbs = moved / dt / 1e9
+    sample = f"first {n_sample} of {lay.padded_numel} arena elements per step, all {K} workers"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic", "params_per_s": n_sample * args.steps / dt,
+        "config": {"workload": wl_name, "layout": wl["layout"], "workers": K, "delay_k": wl["k"],
+                   "grad_dtype": "f32", "sample": sample},
+        "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=4)
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=4)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--threads", type=int, default=0, help="threads per block (0 = library default)")
+    ap.add_argument("--blocks-per-sm", type=int, default=0, help="resident blocks per SM (0 = default)")
+    args = ap.parse_args()
+    wl_name, wl = args.workload, WORKLOADS[args.workload]
+
+    world, rank, local = dist_setup(args.gpus)
+    if args.impl == "reference":
+        if rank == 0:
+            run_reference(args, wl_name, wl)
+        return
+
+    from paper_2012_05396_b200 import binding as B
+    from paper_2012_05396_b200 import build as libbuild
+    from paper_2012_05396_b200 import synth
+    from paper_2012_05396_b200.state import DeviceState
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU path")
+    if rank == 0:
+        libbuild.build_library()
+    torch.cuda.set_device(local)
+    dev_name = f"cuda:{local}"
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(dev_name))
+        dist.barrier()
+
+    K, sg = wl["K"], 4
+    lay = synth.get_layout(wl["layout"])
+    N = lay.padded_numel
+    n_sets = 2
+    need = ((2 + 3 * K) * N * 4 + n_sets * K * N * sg) * 1.05
+    free, _total = torch.cuda.mem_get_info()
+    if need > free:
+        raise SystemExit(f"workload needs {need / 2**30:.1f} GiB, only {free / 2**30:.1f} GiB free")
+
+    nan = float("nan")
+    hp = B.make_hparams(K, wl["lr"], wl["m"], wl["W"], wl["k"], lr_local=nan, alpha=nan, beta=nan,
+                        rescale=nan, grad_dtype=B.SSD_F32)
+    w0 = synth.init_weights(lay, device=dev_name)
+    st = DeviceState(lay.numels, hp, w0, device=dev_name, fill=0.0)
+    if args.threads or args.blocks_per_sm:
+        st.ctx.ssd_set_launch(args.threads, args.blocks_per_sm)
+    mask = synth.valid_mask(lay, dev_name) if N != lay.numel else None
+    grad_sets = [[synth.gradient(lay, s, i, wl["sigma"], device=dev_name, mask=mask) for i in range(K)]
+                 for s in range(n_sets)]
+    stream = torch.cuda.current_stream()
+
+    # SSD warm-up stage + first GLU call, then the bench's own warm-up steps (all untimed).
+    for n in range(wl["W"] + 1 + max(args.warmup, 3)):
+        st.ctx.ssd_step(grad_sets[n % n_sets])
+    torch.cuda.synchronize()
+
+    flags_of = []
+    it0 = st.ctx.ssd_get_counters()[0]
+    for n in range(args.steps):
+        flags_of.append(st.ctx.ssd_schedule(it0 + n)[1])
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    launches0 = st.ctx.ssd_kernel_launches()
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t_wall = time.perf_counter()
+    ev[0].record(stream)
+    for n in range(args.steps):
+        st.ctx.ssd_step(grad_sets[n % n_sets])
+        ev[n + 1].record(stream)
+    torch.cuda.synchronize()
+    t_wall = time.perf_counter() - t_wall
+    if world > 1:
+        dist.barrier()
+    clocks = sampler.stop()
+    launches = st.ctx.ssd_kernel_launches() - launches0
+
+    total_ms = ev[0].elapsed_time(ev[-1])
+    per_launch_ms = [ev[n].elapsed_time(ev[n + 1]) for n in range(args.steps)]
+    if world > 1:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=dev_name)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    bytes_per_launch = [step_bytes_per_param(K, sg, f) * N for f in flags_of]
+    total_bytes = float(sum(bytes_per_launch)) * world
+    value = total_bytes / (total_ms * 1e-3) / 1e9
+    peak, peak_kind = measured_peak()
+    achieved = (sum(bytes_per_launch) / len(bytes_per_launch)) / (statistics.mean(per_launch_ms) * 1e-3) / 1e9
+    traffic = None
+    if NCU_TRAFFIC["digest"] == kernel_digest() and NCU_TRAFFIC["workload"] == wl_name:
+        traffic = NCU_TRAFFIC["bytes_per_launch"]
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "params_per_s": N * args.steps * world / (total_ms * 1e-3),
+        "frac_of_nominal_8TBs": value / world / NOMINAL_HBM_GBS,
+        "wall_ms_per_step": t_wall / args.steps * 1e3,
+        "config": {"workload": wl_name, "layout": wl["layout"], "params": lay.numel, "tensors": lay.num_tensors,
+                   "workers": K, "delay_k": wl["k"], "ssd_warmup_iters": wl["W"], "grad_dtype": "f32",
+                   "stage": "steps-delay", "kernel": "fused ssd_step", "replicas": world,
+                   "device_bytes": st.bytes() + n_sets * K * N * sg,
+                   "l2": "inputs larger than L2 (no flush needed)"
+                   if st.bytes() > 4 * 126e6 else "L2-resident: not an HBM measurement"},
+        "clocks": clocks,
+        "gpu_launches": launches,
+        "roofline": {"bound": "hbm", "kernel": "step_kernel", "achieved": achieved, "peak": peak,
+                     "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind, "traffic": traffic,
+                     "algorithmic_bytes_per_launch": sum(bytes_per_launch) / len(bytes_per_launch),
+                     "launch_ms": {"mean": statistics.mean(per_launch_ms), "min": min(per_launch_ms),
+                                   "max": max(per_launch_ms)}},
+    }
+
+    # ---- end to end: gradients arrive in pinned host memory, the new global weight is read back ----
+    e2e = None
+    if args.e2e_steps > 0:
+        host_grads = [torch.empty(N, dtype=torch.float32).pin_memory() for _ in range(K)]
+        for i in range(K):
+            host_grads[i].copy_(grad_sets[0][i])
+        host_w = torch.empty(N, dtype=torch.float32).pin_memory()
+        staging = grad_sets[1]
+        st.ctx.ssd_step_host(host_grads, staging, host_w)
+        torch.cuda.synchronize()
+        it0 = st.ctx.ssd_get_counters()[0]
+        e_flags = [st.ctx.ssd_schedule(it0 + n)[1] for n in range(args.e2e_steps)]
+        if world > 1:
+            dist.barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for n in range(args.e2e_steps):
+            st.ctx.ssd_step_host(host_grads, staging, host_w)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        e_ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([e_ms], dtype=torch.float64, device=dev_name)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e_ms = float(t.item())
+        e_bytes = float(sum(step_bytes_per_param(K, sg, f) * N for f in e_flags)) * world
+        e2e = {"value": e_bytes / (e_ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": K * N * sg,
+               "d2h_bytes_per_step": N * 4, "steps": args.e2e_steps, "ms_per_step": e_ms / args.e2e_steps,
+               "call": "ssd_step_host"}
+        del host_grads, host_w
+    line["e2e"] = e2e
+
+    # ---- the CPU oracle on the host cores, bounded sample (rank 0, single GPU runs only) ----
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        n_sample = min(N, 1 << 23)
+        g_host = [[g[:n_sample].cpu().numpy() for g in gs] for gs in grad_sets]
+        w_host = w0[:n_sample].cpu().numpy()
+        o_steps = 2 * wl["k"]
+        dt, moved, params, cores = oracle_sample_run(wl, n_sample, o_steps, g_host, w_host)
+        line["cpu_baseline"] = {
+            "value": moved / dt / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "host_cores": os.cpu_count(), "params_per_s": params / dt, "ms_per_step_sample": dt / o_steps * 1e3,
+            "sample": f"first {n_sample} of {N} arena elements, all {K} workers, {o_steps} delay-stage steps"}
+
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,159 @@
+"""The full-size configurations on the GPU, in the launch shape the benchmark times.
+
+Where the oracle cannot sweep every element in seconds, it follows a sample of arena elements
+through the whole schedule: the update is elementwise in the parameter index, so the oracle run on
+the gathered elements (same hyper-parameters, same gradients at those indices) is the exact
+expected value for those positions of the full-size GPU result.  Samples hold every tensor's first
+and last element, the elements around every padding gap, both ends of the arena and a seeded
+random draw.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2012_05396_b200 import binding as B
+from paper_2012_05396_b200 import synth
+from paper_2012_05396_b200.state import DeviceState
+from tests.gpu_common import assert_same, compare_states, make_hp, oracle_grad
+
+pytestmark = pytest.mark.gpu
+
+
+def sample_indices(lay, n_random=4096, seed=5):
+    N = lay.padded_numel
+    picks = [np.arange(0, min(N, 64)), np.arange(max(0, N - 64), N)]
+    for off, cnt in zip(lay.offsets, lay.numels):
+        edge = np.array([off, off + 1, off + cnt - 2, off + cnt - 1, off + cnt, off + cnt + 1, off - 1])
+        picks.append(edge[(edge >= 0) & (edge < N)])
+    picks.append(np.random.default_rng(seed).integers(0, N, n_random))
+    return np.unique(np.concatenate(picks)).astype(np.int64)
+
+
+def run_sampled(layout_name, K, W, k, iters, sigma, lr, m):
+    lay = synth.get_layout(layout_name)
+    ohp, chp = make_hp(K, lr, m, W, k)
+    idx = sample_indices(lay)
+    tidx = torch.from_numpy(idx)
+    w0 = synth.init_weights(lay, device="cuda")
+    dev = DeviceState(lay.numels, chp, w0)
+    ref = oracle.State(ohp, w0[tidx.cuda()].cpu().numpy())
+    mask = synth.valid_mask(lay, "cuda") if lay.padded_numel != lay.numel else None
+    for n in range(iters):
+        grads = [synth.gradient(lay, n, i, sigma, device="cuda", mask=mask) for i in range(K)]
+        dev.ctx.ssd_step(grads)
+        ref.step([synth.gradient_at(lay, n, i, sigma, tidx).numpy() for i in range(K)])
+        del grads
+    torch.cuda.synchronize()
+    compare_states(dev, ref, f"{layout_name} K={K} k={k}", idx=idx)
+    assert dev.ctx.ssd_kernel_launches() == iters
+    # the sample really is the full-size run's data: weights of the sampled positions came from
+    # the device arena, gradients from the same counter-based stream
+    g = synth.gradient(lay, 0, 0, sigma, device="cuda", mask=mask)
+    assert torch.equal(g[tidx.cuda()].cpu(), synth.gradient_at(lay, 0, 0, sigma, tidx))
+
+
+def test_config_resnet50_K8_every_element():
+    # ResNet-50 layout (25.6M parameters, 161 tensors), K=8, sigma 1e-3, W=8, k=4, 50 iterations
+    lay = synth.get_layout("resnet50")
+    K, W, k, iters = 8, 8, 4, 50
+    ohp, chp = make_hp(K, 0.1, 0.9, W, k)
+    w0 = synth.init_weights(lay, device="cuda")
+    dev = DeviceState(lay.numels, chp, w0)
+    ref = oracle.State(ohp, w0.cpu().numpy())
+    for n in range(iters):
+        grads = [synth.gradient(lay, n, i, 1e-3, device="cuda") for i in range(K)]
+        dev.ctx.ssd_step(grads)
+        ref.step([g.cpu().numpy() for g in grads])
+        if n in (W - 1, W, W + k - 1, W + k):
+            torch.cuda.synchronize()
+            compare_states(dev, ref, f"resnet50 iter {n}")
+    torch.cuda.synchronize()
+    compare_states(dev, ref, "resnet50 final")
+
+
+@pytest.mark.parametrize("k", [2, 8])
+def test_config_resnet50_K8_other_delays_sampled(k):
+    run_sampled("resnet50", 8, 8, k, 50, 1e-3, 0.1, 0.9)
+
+
+def test_config_vgg16_K16_sampled():
+    # VGG-16 layout (138M parameters), K=16, sigma 1e-3, lr 0.01, m 0.9, W=4, k=4, 20 iterations:
+    # the workload and launch shape bench.py times
+    need = (2 + 4 * 16) * 138357544 * 4 * 1.1
+    if torch.cuda.mem_get_info()[0] < need:
+        pytest.skip("not enough free device memory for the VGG-16 K=16 state")
+    run_sampled("vgg16", 16, 4, 4, 20, 1e-3, 0.01, 0.9)
+
+
+def prime(n, K, bf16, device, idx=None):
+    """uniform(-1,1) state and gradients of the bandwidth sweep; at `idx` only when given."""
+    def buf(stream, worker=0):
+        if idx is None:
+            return synth.uniform_buffer(stream, n, worker=worker, device=device)
+        return synth.uniform_at(synth.stream_key(synth.SEED, stream, 0, worker), idx)
+    d = dict(w=buf(synth.STREAM_WEIGHT), mom=buf(synth.STREAM_MOM),
+             w_loc=[buf(synth.STREAM_WLOC, i) for i in range(K)],
+             pre=[buf(synth.STREAM_PRE, i) for i in range(K)],
+             g=[buf(synth.STREAM_GRAD, i) for i in range(K)])
+    if bf16:
+        d["g"] = [synth.to_bf16(g) for g in d["g"]]
+    return d
+
+
+def sweep_point(n, K, bf16, glu_flags, sampled):
+    ohp, chp = make_hp(K, 0.1, 0.9, 0, 4, bf16=bf16)
+    idx = None
+    if sampled:
+        idx = np.unique(np.concatenate([np.arange(64), np.arange(n - 64, n),
+                                        np.random.default_rng(n + K).integers(0, n, 4096)])).astype(np.int64)
+    d = prime(n, K, bf16, "cuda")
+    dev = DeviceState([n], chp, d["w"])
+    dev.mom.copy_(d["mom"])
+    for i in range(K):
+        dev.w_loc[i].copy_(d["w_loc"][i]); dev.pre[i].copy_(d["pre"][i])
+    h = prime(n, K, bf16, "cpu", None if idx is None else torch.from_numpy(idx)) if sampled else None
+    def host(name, i=None):
+        t = (h if sampled else d)[name]
+        t = t if i is None else t[i]
+        return oracle_grad(t, bf16) if name == "g" else t.cpu().numpy().copy()
+    ref = oracle.State(ohp, host("w"))
+    ref.mom[:] = host("mom")
+    for i in range(K):
+        ref.w_loc[i][:] = host("w_loc", i); ref.pre[i][:] = host("pre", i)
+    # one synchronous server update, then one GLU update per worker
+    dev.ctx.ssd_server_sync_update(d["g"])
+    oracle.server_update(ohp, [host("g", i) for i in range(K)], ref.w, ref.mom)
+    for i in range(K):
+        dev.ctx.ssd_worker_glu_update(i, d["g"][i], glu_flags)
+        oracle.glu_update(ohp, host("g", i), ref.w_loc[i], ref.pre[i], ref.w_dev[i], ref.w, glu_flags)
+    torch.cuda.synchronize()
+    tag = f"sweep n={n} K={K} bf16={bf16} flags={glu_flags}"
+    assert_same(dev.w, ref.w, tag + " w", idx)
+    assert_same(dev.mom, ref.mom, tag + " mom", idx)
+    for i in range(K):
+        for name in ("w_loc", "pre", "w_dev"):
+            assert_same(getattr(dev, name)[i], getattr(ref, name)[i], f"{tag} {name}[{i}]", idx)
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+@pytest.mark.parametrize("K", [1, 4, 16, 32])
+def test_sweep_points_every_element(K, bf16):
+    for n in (1 << 16, 1 << 20):
+        sweep_point(n, K, bf16, 0, sampled=False)
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_sweep_refresh_and_pull_variants(bf16):
+    sweep_point(1 << 22, 4, bf16, B.SSD_FLAG_REFRESH, sampled=False)
+    sweep_point(1 << 22, 4, bf16, B.SSD_FLAG_PULL, sampled=False)
+    sweep_point(1 << 26, 4, bf16, B.SSD_FLAG_REFRESH | B.SSD_FLAG_PULL, sampled=True)
+
+
+@pytest.mark.parametrize("K,bf16", [(4, False), (32, True), (32, False)])
+def test_sweep_largest_size_sampled(K, bf16):
+    n = 1 << 28
+    need = ((2 + 3 * K) * 4 + K * (2 if bf16 else 4)) * n * 1.1 + (4 << 30)
+    if torch.cuda.mem_get_info()[0] < need:
+        pytest.skip(f"needs {need / 2**30:.0f} GiB of free device memory")
+    sweep_point(n, K, bf16, 0, sampled=True)
