@@ -13,7 +13,8 @@
  *
  * Conventions
  *  - Every pointer in ssd_buffers and every gradient pointer is DEVICE memory
- *    owned by the caller, 16-byte aligned, holding at least ssd_arena_numel()
+ *    owned by the caller, 16-byte aligned (32-byte alignment of every buffer
+ *    enables the 256-bit access path), holding at least ssd_arena_numel()
  *    elements.  The library never allocates, frees or retains device memory of
  *    its own; a context holds host-side metadata only.  Pointer *tables*
  *    (w_loc, pre, w_dev, grads) are HOST arrays of K device pointers and are
@@ -102,7 +103,9 @@ typedef struct {
 } ssd_hparams;
 
 /* Caller-owned device state.  w_loc, pre, w_dev: host arrays of K device pointers.
- * The K*3+2 buffers must not overlap each other or any gradient buffer. */
+ * The K*3+2 buffers must not overlap each other or any gradient buffer.  With
+ * delay_k == 0 (synchronous SGD only) no worker state is ever touched and the
+ * three tables may be NULL. */
 typedef struct {
     float *w;                     /* global weight w_t (server)                 */
     float *mom;                   /* server momentum mom_t                      */
@@ -125,8 +128,10 @@ ssd_status ssd_arena_numel(const ssd_layout *layout, int64_t *padded_numel);
  * Does not touch any buffer.  Before the first step the caller sets w = w_0,
  * mom = 0 and, when warmup_iters == 0, also w_loc[i] = w_0 for every worker
  * (Algorithm 1 starts by pulling w_0); ssd_broadcast_weights does the latter.
- * Errors: SSD_ERR_ARG, SSD_ERR_ALIGN, SSD_ERR_LAYOUT, SSD_ERR_NOMEM, and
- * SSD_ERR_CUDA when no CUDA device is usable.  *out is NULL on error. */
+ * Needs no CUDA device: the current device is looked up at the first launch,
+ * and launching calls return SSD_ERR_CUDA when none is usable.
+ * Errors: SSD_ERR_ARG, SSD_ERR_ALIGN, SSD_ERR_LAYOUT, SSD_ERR_NOMEM.  *out is
+ * NULL on error. */
 ssd_status ssd_init(ssd_ctx **out, const ssd_layout *layout, const ssd_hparams *hp,
                     const ssd_buffers *buffers);
 
@@ -198,7 +203,8 @@ ssd_status ssd_step_host(ssd_ctx *ctx, const void *const *host_grads, void *cons
                          float *host_w_out, void *cuda_stream);
 
 /* w_loc[i] = w for every worker (the initial pull of Algorithm 1).  Needed before
- * the first step only when warmup_iters == 0.  One kernel launch. */
+ * the first step only when warmup_iters == 0.  One kernel launch.  SSD_ERR_STATE
+ * when the context was created without worker state. */
 ssd_status ssd_broadcast_weights(ssd_ctx *ctx, void *cuda_stream);
 
 /* Where worker `worker` finds the weights for its next forward/backward pass
@@ -225,9 +231,18 @@ ssd_status ssd_set_lr(ssd_ctx *ctx, float lr, float lr_local);
 /* Resolved hyper-parameters as the kernels use them, and the derived c. */
 ssd_status ssd_get_hparams(const ssd_ctx *ctx, ssd_hparams *resolved, float *sync_scale);
 
-/* Launch shape of the streaming kernels: threads per block (multiple of 32,
- * 64..1024) and resident blocks per SM (1..32).  0 keeps the default. */
+/* Launch shape of every kernel of this context: threads per block (multiple of
+ * 32, 64..512) and resident blocks per SM (1..32, capped at what fits).  0 for
+ * either returns it to the per-kernel default, which depends on the kernel, K,
+ * the gradient type and the iteration's flags.  Results do not depend on it. */
 ssd_status ssd_set_launch(ssd_ctx *ctx, int32_t threads_per_block, int32_t blocks_per_sm);
+
+/* Shape of the kernels' inner loop.  vector_elems: elements each thread owns per
+ * trip, 8 (256-bit accesses; used only when every buffer involved is 32-byte
+ * aligned, else 4 is taken) or 4 (128-bit); batch: workers whose loads a thread
+ * issues together, 1, 2, 4 or 8 (the fused step uses at most 4).  0 = choose from
+ * the alignment and K.  Results do not depend on either. */
+ssd_status ssd_set_kernel_shape(ssd_ctx *ctx, int32_t vector_elems, int32_t batch);
 
 /* Number of kernels this context has launched so far. */
 int64_t ssd_kernel_launches(const ssd_ctx *ctx);

@@ -15,7 +15,8 @@ from typing import List, Optional, Sequence
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libssd_sgd.so")
+# SSD_SGD_LIBRARY selects another build of the same library (e.g. one compiled with other cache hints)
+LIB_PATH = os.environ.get("SSD_SGD_LIBRARY") or os.path.join(_HERE, "libssd_sgd.so")
 
 SSD_OK, SSD_ERR_ARG, SSD_ERR_ALIGN, SSD_ERR_LAYOUT, SSD_ERR_STATE, SSD_ERR_CUDA, SSD_ERR_NOMEM = range(7)
 SSD_F32, SSD_BF16 = 0, 1
@@ -28,7 +29,8 @@ EXPORTS = (
     "ssd_arena_numel", "ssd_init", "ssd_destroy", "ssd_tensor_offset", "ssd_schedule",
     "ssd_server_sync_update", "ssd_worker_glu_update", "ssd_worker_local_step", "ssd_advance",
     "ssd_step", "ssd_step_host", "ssd_broadcast_weights", "ssd_worker_weights", "ssd_get_counters",
-    "ssd_set_counters", "ssd_set_lr", "ssd_get_hparams", "ssd_set_launch", "ssd_kernel_launches",
+    "ssd_set_counters", "ssd_set_lr", "ssd_get_hparams", "ssd_set_launch", "ssd_set_kernel_shape",
+    "ssd_kernel_launches",
     "ssd_status_str", "ssd_last_cuda_error",
 )
 
@@ -88,6 +90,7 @@ def lib():
             "ssd_set_lr": (i32, [vp, C.c_float, C.c_float]),
             "ssd_get_hparams": (i32, [vp, P(ssd_hparams), P(C.c_float)]),
             "ssd_set_launch": (i32, [vp, i32, i32]),
+            "ssd_set_kernel_shape": (i32, [vp, i32, i32]),
             "ssd_kernel_launches": (i64, [vp]),
             "ssd_status_str": (C.c_char_p, [i32]),
             "ssd_last_cuda_error": (C.c_char_p, [vp]),
@@ -144,13 +147,14 @@ def make_hparams(K: int, lr: float, momentum: float, warmup_iters: int, delay_k:
 class Context:
     """Owner of one ssd_ctx handle.  Methods carry the names of the C entry points."""
 
-    def __init__(self, numels: Sequence[int], hp: ssd_hparams, w, mom, w_loc: Sequence, pre: Sequence,
-                 w_dev: Sequence):
+    def __init__(self, numels: Sequence[int], hp: ssd_hparams, w, mom, w_loc: Optional[Sequence] = None,
+                 pre: Optional[Sequence] = None, w_dev: Optional[Sequence] = None):
         self._h = C.c_void_p()
         self.K = hp.K
-        self._keep = (w, mom, list(w_loc), list(pre), list(w_dev))      # keep tensors alive
+        self._keep = (w, mom, w_loc, pre, w_dev)                         # keep tensors alive
         lay, _arr = _layout(numels)
-        bufs = ssd_buffers(_ptr(w), _ptr(mom), _ptr_table(w_loc), _ptr_table(pre), _ptr_table(w_dev))
+        tables = [None if t is None else _ptr_table(t) for t in (w_loc, pre, w_dev)]
+        bufs = ssd_buffers(_ptr(w), _ptr(mom), *tables)
         st = lib().ssd_init(C.byref(self._h), C.byref(lay), C.byref(hp), C.byref(bufs))
         if st != SSD_OK:
             self._h = C.c_void_p()
@@ -233,6 +237,9 @@ class Context:
 
     def ssd_set_launch(self, threads_per_block: int = 0, blocks_per_sm: int = 0):
         self._check(lib().ssd_set_launch(self._h, threads_per_block, blocks_per_sm), "ssd_set_launch")
+
+    def ssd_set_kernel_shape(self, vector_elems: int = 0, batch: int = 0):
+        self._check(lib().ssd_set_kernel_shape(self._h, vector_elems, batch), "ssd_set_kernel_shape")
 
     def ssd_kernel_launches(self) -> int:
         return lib().ssd_kernel_launches(self._h)

@@ -8,8 +8,9 @@
 //                 element is read once and feeds the server sum and its own
 //                 worker's GLU update
 // All three are bound by HBM bandwidth (well under one flop per byte), so the
-// design is about bytes: 128-bit loads and stores, every byte touched once,
-// streaming cache hints, several independent loads in flight per thread.
+// design is about bytes: every byte touched once, 256-bit (or 128-bit) fully
+// coalesced accesses, streaming cache hints, and enough independent loads in
+// flight per SM to cover the DRAM latency.
 //
 // Arithmetic contract: binary32, round to nearest, every operation rounded on
 // its own.  The __f*_rn intrinsics are never contracted into fused multiply-adds,
@@ -18,6 +19,18 @@
 
 #include <cuda_runtime.h>
 #include <stdint.h>
+
+// Cache policy of the streaming accesses (PTX qualifiers).  State and gradients
+// are far larger than L2 and each byte is used once per kernel: evict-first.
+#ifndef SSD_LD_QUAL
+#define SSD_LD_QUAL ".cs"
+#endif
+#ifndef SSD_LDG_QUAL
+#define SSD_LDG_QUAL ".cs"
+#endif
+#ifndef SSD_ST_QUAL
+#define SSD_ST_QUAL ".cs"
+#endif
 
 namespace ssd {
 
@@ -69,37 +82,95 @@ struct CopyParams {
 };
 
 // ---------------------------------------------------------------------------
-// VW consecutive elements; VW = 4 is one 128-bit access.  Arena lengths are
-// multiples of 4 elements by construction, so there is no ragged tail.
+// VW consecutive elements owned by one thread: VW = 8 is one 256-bit access to
+// float32 data (sm_100 has 256-bit global loads and stores) and one 128-bit
+// access to bfloat16 data; VW = 4 is the 128-bit / 64-bit form for buffers that
+// are only 16-byte aligned, and finishes a length that is not a multiple of 8.
 // ---------------------------------------------------------------------------
 template <int VW> struct Vec { float v[VW]; };
 
-template <int VW> __device__ __forceinline__ Vec<VW> ld_f32(const float *p, int64_t e);
-template <> __device__ __forceinline__ Vec<4> ld_f32<4>(const float *p, int64_t e)
-{
-    float4 t = __ldcs(reinterpret_cast<const float4 *>(p + e));
-    return Vec<4>{{t.x, t.y, t.z, t.w}};
-}
+// Loads of VW float32 values with a given cache qualifier.
+#define SSD_DEFINE_LD_F32(NAME, QUAL)                                                           \
+    template <int VW> __device__ __forceinline__ Vec<VW> NAME(const float *p, int64_t e);       \
+    template <> __device__ __forceinline__ Vec<4> NAME<4>(const float *p, int64_t e)            \
+    {                                                                                           \
+        Vec<4> r;                                                                               \
+        asm volatile("ld.global" QUAL ".v4.f32 {%0,%1,%2,%3}, [%4];"                            \
+                     : "=f"(r.v[0]), "=f"(r.v[1]), "=f"(r.v[2]), "=f"(r.v[3])                   \
+                     : "l"(p + e));                                                             \
+        return r;                                                                               \
+    }                                                                                           \
+    template <> __device__ __forceinline__ Vec<8> NAME<8>(const float *p, int64_t e)            \
+    {                                                                                           \
+        Vec<8> r;                                                                               \
+        asm volatile("ld.global" QUAL ".v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"                \
+                     : "=f"(r.v[0]), "=f"(r.v[1]), "=f"(r.v[2]), "=f"(r.v[3]), "=f"(r.v[4]),    \
+                       "=f"(r.v[5]), "=f"(r.v[6]), "=f"(r.v[7])                                 \
+                     : "l"(p + e));                                                             \
+        return r;                                                                               \
+    }
+
+SSD_DEFINE_LD_F32(ld_f32, SSD_LD_QUAL)        // state: read, then overwritten by the same thread
+SSD_DEFINE_LD_F32(ld_f32_ro, SSD_LDG_QUAL)    // gradients: read-only for the whole kernel
 
 template <int VW> __device__ __forceinline__ void st_f32(float *p, int64_t e, const Vec<VW> &x);
 template <> __device__ __forceinline__ void st_f32<4>(float *p, int64_t e, const Vec<4> &x)
 {
-    __stcs(reinterpret_cast<float4 *>(p + e), make_float4(x.v[0], x.v[1], x.v[2], x.v[3]));
+    asm volatile("st.global" SSD_ST_QUAL ".v4.f32 [%0], {%1,%2,%3,%4};" ::"l"(p + e), "f"(x.v[0]),
+                 "f"(x.v[1]), "f"(x.v[2]), "f"(x.v[3])
+                 : "memory");
+}
+template <> __device__ __forceinline__ void st_f32<8>(float *p, int64_t e, const Vec<8> &x)
+{
+    asm volatile("st.global" SSD_ST_QUAL ".v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p + e),
+                 "f"(x.v[0]), "f"(x.v[1]), "f"(x.v[2]), "f"(x.v[3]), "f"(x.v[4]), "f"(x.v[5]),
+                 "f"(x.v[6]), "f"(x.v[7])
+                 : "memory");
 }
 
 __device__ __forceinline__ float bf16_lo(uint32_t pair) { return __uint_as_float(pair << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t pair) { return __uint_as_float(pair & 0xffff0000u); }
 
-// Gradient load: float32 as is, bfloat16 widened exactly (bits << 16).
-template <int GT, int VW> __device__ __forceinline__ Vec<VW> ld_grad(const void *p, int64_t e);
-template <> __device__ __forceinline__ Vec<4> ld_grad<kF32, 4>(const void *p, int64_t e)
+// A gradient vector as loaded: float32 values, or bfloat16 kept packed two per
+// register until they are used (a load in flight then costs one register per four
+// bytes for either type).  get(l) widens bfloat16 exactly (bits << 16).
+template <int GT, int VW> struct Grad;
+template <int VW> struct Grad<kF32, VW> {
+    Vec<VW> raw;
+    __device__ __forceinline__ float get(int l) const { return raw.v[l]; }
+};
+template <int VW> struct Grad<kBF16, VW> {
+    uint32_t raw[VW / 2];
+    __device__ __forceinline__ float get(int l) const
+    {
+        return (l & 1) ? bf16_hi(raw[l >> 1]) : bf16_lo(raw[l >> 1]);
+    }
+};
+
+template <int GT, int VW> __device__ __forceinline__ Grad<GT, VW> ld_grad(const void *p, int64_t e);
+template <> __device__ __forceinline__ Grad<kF32, 4> ld_grad<kF32, 4>(const void *p, int64_t e)
 {
-    return ld_f32<4>(static_cast<const float *>(p), e);
+    return Grad<kF32, 4>{ld_f32_ro<4>(static_cast<const float *>(p), e)};
 }
-template <> __device__ __forceinline__ Vec<4> ld_grad<kBF16, 4>(const void *p, int64_t e)
+template <> __device__ __forceinline__ Grad<kF32, 8> ld_grad<kF32, 8>(const void *p, int64_t e)
 {
-    uint2 t = __ldcs(reinterpret_cast<const uint2 *>(static_cast<const uint16_t *>(p) + e));
-    return Vec<4>{{bf16_lo(t.x), bf16_hi(t.x), bf16_lo(t.y), bf16_hi(t.y)}};
+    return Grad<kF32, 8>{ld_f32_ro<8>(static_cast<const float *>(p), e)};
+}
+template <> __device__ __forceinline__ Grad<kBF16, 4> ld_grad<kBF16, 4>(const void *p, int64_t e)
+{
+    Grad<kBF16, 4> r;
+    asm volatile("ld.global" SSD_LDG_QUAL ".v2.u32 {%0,%1}, [%2];"
+                 : "=r"(r.raw[0]), "=r"(r.raw[1])
+                 : "l"(static_cast<const uint16_t *>(p) + e));
+    return r;
+}
+template <> __device__ __forceinline__ Grad<kBF16, 8> ld_grad<kBF16, 8>(const void *p, int64_t e)
+{
+    Grad<kBF16, 8> r;
+    asm volatile("ld.global" SSD_LDG_QUAL ".v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.raw[0]), "=r"(r.raw[1]), "=r"(r.raw[2]), "=r"(r.raw[3])
+                 : "l"(static_cast<const uint16_t *>(p) + e));
+    return r;
 }
 
 // ---------------------------------------------------------------------------
@@ -140,7 +211,7 @@ __device__ __forceinline__ void sync_at(const SyncParams &p, int64_t e)
     Vec<VW> mom = ld_f32<VW>(p.mom, e);
     Vec<VW> sum;
     for (int i0 = 0; i0 < p.K; i0 += B) {
-        Vec<VW> g[B];
+        Grad<GT, VW> g[B];
 #pragma unroll
         for (int b = 0; b < B; ++b)
             if (i0 + b < p.K) g[b] = ld_grad<GT, VW>(p.g[i0 + b], e);
@@ -149,7 +220,7 @@ __device__ __forceinline__ void sync_at(const SyncParams &p, int64_t e)
             if (i0 + b < p.K) {
 #pragma unroll
                 for (int l = 0; l < VW; ++l)
-                    sum.v[l] = (i0 + b == 0) ? g[b].v[l] : __fadd_rn(sum.v[l], g[b].v[l]);
+                    sum.v[l] = (i0 + b == 0) ? g[b].get(l) : __fadd_rn(sum.v[l], g[b].get(l));
             }
         }
     }
@@ -165,14 +236,14 @@ template <int GT, int VW>
 __device__ __forceinline__ void glu_at(const GluParams &p, int64_t e)
 {
     const bool first = p.flags & kFirst, refresh = p.flags & kRefresh, pull = p.flags & kPull;
-    Vec<VW> g = ld_grad<GT, VW>(p.g, e);
+    Grad<GT, VW> g = ld_grad<GT, VW>(p.g, e);
     Vec<VW> wl = ld_f32<VW>(p.w_loc, e);
     Vec<VW> pr = first ? wl : ld_f32<VW>(p.pre, e);
     Vec<VW> wg;
     if (pull) wg = ld_f32<VW>(p.w, e);
     Vec<VW> r;
 #pragma unroll
-    for (int l = 0; l < VW; ++l) r.v[l] = glu_elem(g.v[l], wl.v[l], pr.v[l], p.s);
+    for (int l = 0; l < VW; ++l) r.v[l] = glu_elem(g.get(l), wl.v[l], pr.v[l], p.s);
     if (first || refresh) st_f32<VW>(p.pre, e, wl);
     if (pull) {
         st_f32<VW>(p.w_dev, e, r);
@@ -190,7 +261,8 @@ __device__ __forceinline__ void step_at(const StepParams &p, int64_t e)
     Vec<VW> mom = ld_f32<VW>(p.mom, e);
     Vec<VW> sum;
     for (int i0 = 0; i0 < p.K; i0 += B) {
-        Vec<VW> g[B], wl[B], pr[B];
+        Grad<GT, VW> g[B];
+        Vec<VW> wl[B], pr[B];
 #pragma unroll
         for (int b = 0; b < B; ++b) {
             if (i0 + b < p.K) {
@@ -206,8 +278,9 @@ __device__ __forceinline__ void step_at(const StepParams &p, int64_t e)
                 Vec<VW> r;
 #pragma unroll
                 for (int l = 0; l < VW; ++l) {
-                    sum.v[l] = (i == 0) ? g[b].v[l] : __fadd_rn(sum.v[l], g[b].v[l]);
-                    r.v[l] = glu_elem(g[b].v[l], wl[b].v[l], first ? wl[b].v[l] : pr[b].v[l], p.s);
+                    const float gl = g[b].get(l);
+                    sum.v[l] = (i == 0) ? gl : __fadd_rn(sum.v[l], gl);
+                    r.v[l] = glu_elem(gl, wl[b].v[l], first ? wl[b].v[l] : pr[b].v[l], p.s);
                 }
                 if (first || refresh) st_f32<VW>(p.pre[i], e, wl[b]);
                 st_f32<VW>(pull ? p.w_dev[i] : p.w_loc[i], e, r);
@@ -223,43 +296,53 @@ __device__ __forceinline__ void step_at(const StepParams &p, int64_t e)
 }
 
 // ---------------------------------------------------------------------------
-// Kernels: grid-stride over the n/4 128-bit vectors of the arena.
+// Kernels: grid-stride over the n/VW vectors of the arena.  Arena lengths are
+// multiples of 4; with VW = 8 a remainder of 4 elements is finished by one
+// thread with the 128-bit body.
 // ---------------------------------------------------------------------------
-#define SSD_SWEEP(n, BODY)                                                                \
+#define SSD_SWEEP(n, VW, BODY, TAIL)                                                      \
     do {                                                                                  \
-        const int64_t nvec = (n) >> 2;                                                    \
+        const int64_t nvec = (n) / (VW);                                                  \
         const int64_t stride = (int64_t)gridDim.x * blockDim.x;                           \
         for (int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; v < nvec; v += stride) { \
-            const int64_t e = v << 2;                                                     \
+            const int64_t e = v * (VW);                                                   \
             BODY;                                                                         \
+        }                                                                                 \
+        if ((VW) == 8 && blockIdx.x == 0 && threadIdx.x == 0 && nvec * (VW) < (n)) {      \
+            const int64_t e = nvec * (VW);                                                \
+            TAIL;                                                                         \
         }                                                                                 \
     } while (0)
 
-template <int GT, int B>
+template <int GT, int VW, int B>
 __global__ void __launch_bounds__(kMaxThreads) sync_kernel(const __grid_constant__ SyncParams p)
 {
-    SSD_SWEEP(p.n, (sync_at<GT, 4, B>(p, e)));
+    SSD_SWEEP(p.n, VW, (sync_at<GT, VW, B>(p, e)), (sync_at<GT, 4, B>(p, e)));
 }
 
-template <int GT>
+template <int GT, int VW>
 __global__ void __launch_bounds__(kMaxThreads) glu_kernel(const __grid_constant__ GluParams p)
 {
-    SSD_SWEEP(p.n, (glu_at<GT, 4>(p, e)));
+    SSD_SWEEP(p.n, VW, (glu_at<GT, VW>(p, e)), (glu_at<GT, 4>(p, e)));
 }
 
-template <int GT, int B>
+template <int GT, int VW, int B>
 __global__ void __launch_bounds__(kMaxThreads) step_kernel(const __grid_constant__ StepParams p)
 {
-    SSD_SWEEP(p.n, (step_at<GT, 4, B>(p, e)));
+    SSD_SWEEP(p.n, VW, (step_at<GT, VW, B>(p, e)), (step_at<GT, 4, B>(p, e)));
+}
+
+template <int VW> __device__ __forceinline__ void copy_at(const CopyParams &p, int64_t e)
+{
+    Vec<VW> x = ld_f32<VW>(p.src, e);
+    for (int i = 0; i < p.K; ++i) st_f32<VW>(p.dst[i], e, x);
 }
 
 // dst[i] = src for K destinations (the pull of a freshly initialised or warm-up weight).
+template <int VW>
 __global__ void __launch_bounds__(kMaxThreads) copy_kernel(const __grid_constant__ CopyParams p)
 {
-    SSD_SWEEP(p.n, {
-        Vec<4> x = ld_f32<4>(p.src, e);
-        for (int i = 0; i < p.K; ++i) st_f32<4>(p.dst[i], e, x);
-    });
+    SSD_SWEEP(p.n, VW, (copy_at<VW>(p, e)), (copy_at<4>(p, e)));
 }
 
 }  // namespace ssd

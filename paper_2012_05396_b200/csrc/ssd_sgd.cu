@@ -31,8 +31,11 @@ struct ssd_ctx {
     Scalars s{};
     float *w = nullptr, *mom = nullptr;
     float *w_loc[kMaxWorkers]{}, *pre[kMaxWorkers]{}, *w_dev[kMaxWorkers]{};
+    bool has_workers = true;          // false: delay_k == 0 and no worker tables were given
     int64_t iter = 0, loc_update = 0;
-    int threads = 256, blocks_per_sm = 0;   // 0: as many as fit (occupancy query)
+    bool state32 = false;             // every state buffer is 32-byte aligned
+    int threads = 0, blocks_per_sm = 0;     // 0: the kernel's default shape
+    int force_vw = 0, force_batch = 0;      // 0: chosen from alignment and K
     int64_t launches = 0;
     Device dev;
     std::string cuda_error;
@@ -105,19 +108,24 @@ ssd_status ensure_device(ssd_ctx *c)
     return SSD_OK;
 }
 
-// Grid for a sweep over n elements: one 128-bit vector per thread per trip, at most
-// `blocks_per_sm` resident blocks per SM so that the grid is one full wave.
+// Launch shape of one sweep: elements per thread per trip, workers whose loads are issued
+// together, threads per block, resident blocks per SM (0 = as many as fit).
+struct Shape {
+    int vw, batch, threads, per_sm;
+};
+
+// Grid for a sweep over n elements: at most `per_sm` resident blocks per SM, never more than
+// fit, so that the grid is a single wave and every block's trips are equally long.
 template <typename Kernel>
-ssd_status grid_for(ssd_ctx *c, Kernel kernel, int64_t n, int *grid)
+ssd_status grid_for(ssd_ctx *c, Kernel kernel, int64_t n, const Shape &sh, int *grid)
 {
-    int per_sm = c->blocks_per_sm;
-    if (per_sm == 0) {
-        cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, c->threads, 0);
-        if (e != cudaSuccess) return cuda_fail(c, e);
-        if (per_sm < 1) per_sm = 1;
-    }
-    const int64_t nvec = n >> 2;
-    int64_t need = (nvec + c->threads - 1) / c->threads;
+    int fit = 0;
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&fit, kernel, sh.threads, 0);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    if (fit < 1) fit = 1;
+    const int per_sm = (sh.per_sm > 0 && sh.per_sm < fit) ? sh.per_sm : fit;
+    const int64_t nvec = n / sh.vw;
+    int64_t need = (nvec + sh.threads - 1) / sh.threads;
     if (need < 1) need = 1;
     const int64_t wave = static_cast<int64_t>(c->dev.sms) * per_sm;
     *grid = static_cast<int>(need < wave ? need : wave);
@@ -125,22 +133,79 @@ ssd_status grid_for(ssd_ctx *c, Kernel kernel, int64_t n, int *grid)
 }
 
 template <typename Kernel, typename Params>
-ssd_status launch(ssd_ctx *c, Kernel kernel, const Params &p, int64_t n, cudaStream_t stream)
+ssd_status launch(ssd_ctx *c, Kernel kernel, const Params &p, int64_t n, const Shape &sh, cudaStream_t stream)
 {
     ssd_status st = ensure_device(c);
     if (st != SSD_OK) return st;
     int grid = 1;
-    st = grid_for(c, kernel, n, &grid);
+    st = grid_for(c, kernel, n, sh, &grid);
     if (st != SSD_OK) return st;
-    kernel<<<grid, c->threads, 0, stream>>>(p);
+    kernel<<<grid, sh.threads, 0, stream>>>(p);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(c, e);
     c->launches += 1;
     return SSD_OK;
 }
 
-constexpr int kSyncBatch = 8;   // gradient loads in flight per thread in sync_kernel
-constexpr int kStepBatch = 4;   // workers (3 loads each) in flight per thread in step_kernel
+bool aligned32(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 31u) == 0; }
+
+// 8 elements per thread (256-bit accesses) need 32-byte aligned float32 buffers; bfloat16
+// gradient buffers are then read 128 bits at a time and need 16 bytes, which every buffer has.
+bool can_use_256bit(const ssd_ctx *c, bool state32, const void *const *grads, int count)
+{
+    if (!state32) return false;
+    if (c->hp.grad_dtype == SSD_F32)
+        for (int i = 0; i < count; ++i)
+            if (!aligned32(grads[i])) return false;
+    return true;
+}
+
+// The caller's overrides (ssd_set_kernel_shape, ssd_set_launch) on top of a default shape.
+Shape finish_shape(const ssd_ctx *c, Shape sh, bool wide_ok, int max_batch)
+{
+    if (c->force_vw) sh.vw = c->force_vw;
+    if (sh.vw == 8 && !wide_ok) sh.vw = 4;
+    if (c->force_batch) sh.batch = c->force_batch;
+    if (sh.batch > max_batch) sh.batch = max_batch;
+    if (c->threads) {
+        sh.threads = c->threads;
+        sh.per_sm = c->blocks_per_sm;
+    } else if (c->blocks_per_sm) {
+        sh.per_sm = c->blocks_per_sm;
+    }
+    return sh;
+}
+
+// Default shapes.  These kernels are limited by how well HBM is kept busy, which depends on
+// the bytes in flight per SM (threads x loads per thread x bytes per load) and on the mix of
+// reads and writes: too few bytes in flight cannot cover the DRAM latency, too many lower
+// the DRAM efficiency again, sooner so when a large share of the traffic is writes.  The
+// values below are the measured optima on B200 (arenas of 25M..138M elements).
+Shape sync_shape(const ssd_ctx *c, bool wide_ok)
+{
+    const int K = c->hp.K;
+    Shape sh;
+    if (c->hp.grad_dtype == SSD_BF16)
+        sh = K >= 4 ? Shape{8, 4, 128, 6} : Shape{8, 1, 128, 4};
+    else
+        sh = K >= 4 ? Shape{8, 4, 128, 5} : Shape{8, 1, 128, 6};
+    return finish_shape(c, sh, wide_ok, 8);
+}
+
+Shape step_shape(const ssd_ctx *c, int flags, bool wide_ok)
+{
+    const int K = c->hp.K;
+    Shape sh;
+    if (flags & (kRefresh | kPull | kFirst))
+        sh = Shape{8, 1, 128, 4};          // write-heavy iterations: 512 threads per SM
+    else if (c->hp.grad_dtype == SSD_BF16)
+        sh = Shape{8, 1, 128, 5};
+    else
+        sh = Shape{8, 1, 128, K >= 16 ? 6 : 5};
+    return finish_shape(c, sh, wide_ok, 4);
+}
+
+Shape glu_shape(const ssd_ctx *c, bool wide_ok) { return finish_shape(c, Shape{8, 1, 256, 0}, wide_ok, 1); }
 
 ssd_status check_grads(const ssd_ctx *c, const void *const *grads)
 {
@@ -150,6 +215,17 @@ ssd_status check_grads(const ssd_ctx *c, const void *const *grads)
         if (!aligned16(grads[i])) return SSD_ERR_ALIGN;
     }
     return SSD_OK;
+}
+
+template <int GT, int VW>
+ssd_status launch_sync_b(ssd_ctx *c, const SyncParams &p, const Shape &sh, cudaStream_t stream)
+{
+    switch (sh.batch) {
+    case 1: return launch(c, sync_kernel<GT, VW, 1>, p, c->n, sh, stream);
+    case 2: return launch(c, sync_kernel<GT, VW, 2>, p, c->n, sh, stream);
+    case 4: return launch(c, sync_kernel<GT, VW, 4>, p, c->n, sh, stream);
+    default: return launch(c, sync_kernel<GT, VW, 8>, p, c->n, sh, stream);
+    }
 }
 
 ssd_status launch_sync(ssd_ctx *c, const void *const *grads, int flags, cudaStream_t stream)
@@ -165,9 +241,12 @@ ssd_status launch_sync(ssd_ctx *c, const void *const *grads, int flags, cudaStre
     p.K = c->hp.K;
     p.flags = flags;
     p.s = c->s;
-    if (c->hp.grad_dtype == SSD_BF16)
-        return launch(c, sync_kernel<kBF16, kSyncBatch>, p, c->n, stream);
-    return launch(c, sync_kernel<kF32, kSyncBatch>, p, c->n, stream);
+    const bool state32 = (flags & kCopy) ? c->state32 : (aligned32(c->w) && aligned32(c->mom));
+    const Shape sh = sync_shape(c, can_use_256bit(c, state32, grads, c->hp.K));
+    const bool bf16 = c->hp.grad_dtype == SSD_BF16;
+    if (sh.vw == 8)
+        return bf16 ? launch_sync_b<kBF16, 8>(c, p, sh, stream) : launch_sync_b<kF32, 8>(c, p, sh, stream);
+    return bf16 ? launch_sync_b<kBF16, 4>(c, p, sh, stream) : launch_sync_b<kF32, 4>(c, p, sh, stream);
 }
 
 ssd_status launch_glu(ssd_ctx *c, int worker, const void *grad, int flags, cudaStream_t stream)
@@ -181,8 +260,23 @@ ssd_status launch_glu(ssd_ctx *c, int worker, const void *grad, int flags, cudaS
     p.n = c->n;
     p.flags = flags;
     p.s = c->s;
-    if (c->hp.grad_dtype == SSD_BF16) return launch(c, glu_kernel<kBF16>, p, c->n, stream);
-    return launch(c, glu_kernel<kF32>, p, c->n, stream);
+    const Shape sh = glu_shape(c, can_use_256bit(c, c->state32, &grad, 1));
+    const bool bf16 = c->hp.grad_dtype == SSD_BF16;
+    if (sh.vw == 8)
+        return bf16 ? launch(c, glu_kernel<kBF16, 8>, p, c->n, sh, stream)
+                    : launch(c, glu_kernel<kF32, 8>, p, c->n, sh, stream);
+    return bf16 ? launch(c, glu_kernel<kBF16, 4>, p, c->n, sh, stream)
+                : launch(c, glu_kernel<kF32, 4>, p, c->n, sh, stream);
+}
+
+template <int GT, int VW>
+ssd_status launch_step_b(ssd_ctx *c, const StepParams &p, const Shape &sh, cudaStream_t stream)
+{
+    switch (sh.batch) {
+    case 1: return launch(c, step_kernel<GT, VW, 1>, p, c->n, sh, stream);
+    case 2: return launch(c, step_kernel<GT, VW, 2>, p, c->n, sh, stream);
+    default: return launch(c, step_kernel<GT, VW, 4>, p, c->n, sh, stream);
+    }
 }
 
 ssd_status launch_step(ssd_ctx *c, const void *const *grads, int flags, cudaStream_t stream)
@@ -200,9 +294,11 @@ ssd_status launch_step(ssd_ctx *c, const void *const *grads, int flags, cudaStre
     p.K = c->hp.K;
     p.flags = flags;
     p.s = c->s;
-    if (c->hp.grad_dtype == SSD_BF16)
-        return launch(c, step_kernel<kBF16, kStepBatch>, p, c->n, stream);
-    return launch(c, step_kernel<kF32, kStepBatch>, p, c->n, stream);
+    const Shape sh = step_shape(c, flags, can_use_256bit(c, c->state32, grads, c->hp.K));
+    const bool bf16 = c->hp.grad_dtype == SSD_BF16;
+    if (sh.vw == 8)
+        return bf16 ? launch_step_b<kBF16, 8>(c, p, sh, stream) : launch_step_b<kF32, 8>(c, p, sh, stream);
+    return bf16 ? launch_step_b<kBF16, 4>(c, p, sh, stream) : launch_step_b<kF32, 4>(c, p, sh, stream);
 }
 
 ssd_status launch_copy(ssd_ctx *c, int first_worker, int count, cudaStream_t stream)
@@ -212,7 +308,9 @@ ssd_status launch_copy(ssd_ctx *c, int first_worker, int count, cudaStream_t str
     p.src = c->w;
     p.n = c->n;
     p.K = count;
-    return launch(c, copy_kernel, p, c->n, stream);
+    const Shape sh = finish_shape(c, Shape{8, 1, 256, 0}, c->state32, 1);
+    if (sh.vw == 8) return launch(c, copy_kernel<8>, p, c->n, sh, stream);
+    return launch(c, copy_kernel<4>, p, c->n, sh, stream);
 }
 
 void advance(ssd_ctx *c)
@@ -248,7 +346,10 @@ ssd_status ssd_init(ssd_ctx **out, const ssd_layout *layout, const ssd_hparams *
     if (std::isinf(hp->lr_local) || std::isinf(hp->alpha) || std::isinf(hp->beta) ||
         std::isinf(hp->rescale))
         return SSD_ERR_ARG;
-    if (!b->w || !b->mom || !b->w_loc || !b->pre || !b->w_dev) return SSD_ERR_ARG;
+    // Without a delay stage (delay_k == 0) no worker state is ever touched: the tables may be NULL.
+    const bool workers = hp->delay_k > 0 || (b->w_loc && b->pre && b->w_dev);
+    if (!b->w || !b->mom) return SSD_ERR_ARG;
+    if (hp->delay_k > 0 && (!b->w_loc || !b->pre || !b->w_dev)) return SSD_ERR_ARG;
 
     ssd_ctx *c = new (std::nothrow) ssd_ctx;
     if (!c) return SSD_ERR_NOMEM;
@@ -258,7 +359,7 @@ ssd_status ssd_init(ssd_ctx **out, const ssd_layout *layout, const ssd_hparams *
         return st;
     }
     std::vector<const void *> all{b->w, b->mom};
-    for (int i = 0; i < hp->K; ++i) {
+    for (int i = 0; workers && i < hp->K; ++i) {
         all.push_back(b->w_loc[i]);
         all.push_back(b->pre[i]);
         all.push_back(b->w_dev[i]);
@@ -292,7 +393,10 @@ ssd_status ssd_init(ssd_ctx **out, const ssd_layout *layout, const ssd_hparams *
     c->s.c = derive_sync_scale(c->hp.lr, c->hp.momentum, c->hp.delay_k);
     c->w = b->w;
     c->mom = b->mom;
-    for (int i = 0; i < hp->K; ++i) {
+    c->has_workers = workers;
+    c->state32 = true;
+    for (const void *p : all) c->state32 = c->state32 && aligned32(p);
+    for (int i = 0; workers && i < hp->K; ++i) {
         c->w_loc[i] = b->w_loc[i];
         c->pre[i] = b->pre[i];
         c->w_dev[i] = b->w_dev[i];
@@ -404,6 +508,7 @@ ssd_status ssd_step_host(ssd_ctx *ctx, const void *const *host_grads, void *cons
 ssd_status ssd_broadcast_weights(ssd_ctx *ctx, void *cuda_stream)
 {
     if (!ctx) return SSD_ERR_ARG;
+    if (!ctx->has_workers) return SSD_ERR_STATE;
     return launch_copy(ctx, 0, ctx->hp.K, static_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -482,6 +587,16 @@ ssd_status ssd_set_launch(ssd_ctx *ctx, int32_t threads_per_block, int32_t block
     if (blocks_per_sm < 0 || blocks_per_sm > 32) return SSD_ERR_ARG;
     if (threads_per_block) ctx->threads = threads_per_block;
     ctx->blocks_per_sm = blocks_per_sm;
+    return SSD_OK;
+}
+
+ssd_status ssd_set_kernel_shape(ssd_ctx *ctx, int32_t vector_elems, int32_t batch)
+{
+    if (!ctx) return SSD_ERR_ARG;
+    if (vector_elems != 0 && vector_elems != 4 && vector_elems != 8) return SSD_ERR_ARG;
+    if (batch != 0 && batch != 1 && batch != 2 && batch != 4 && batch != 8) return SSD_ERR_ARG;
+    ctx->force_vw = vector_elems;
+    ctx->force_batch = batch;
     return SSD_OK;
 }
 

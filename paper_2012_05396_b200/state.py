@@ -16,7 +16,7 @@ class DeviceState:
     """
 
     def __init__(self, numels: Sequence[int], hp: B.ssd_hparams, w0: torch.Tensor,
-                 device="cuda", fill: float = float("nan")):
+                 device="cuda", fill: float = float("nan"), worker_state: bool = True):
         self.numels = [int(n) for n in numels]
         self.n = B.ssd_arena_numel(self.numels)
         assert w0.numel() == self.n and w0.dtype == torch.float32
@@ -24,6 +24,12 @@ class DeviceState:
         self.device = torch.device(device)
         self.w = w0.to(self.device).clone()
         self.mom = torch.zeros(self.n, dtype=torch.float32, device=self.device)
+        if not worker_state:
+            # synchronous SGD only (delay_k == 0): the server state is all there is
+            assert hp.delay_k == 0
+            self.w_loc, self.pre, self.w_dev = [], [], []
+            self.ctx = B.Context(self.numels, hp, self.w, self.mom)
+            return
         # Algorithm 1 starts with every worker pulling w_0.
         self.w_loc = [self.w.clone() for _ in range(self.K)]
         self.pre = [torch.full((self.n,), fill, dtype=torch.float32, device=self.device)
@@ -38,4 +44,4 @@ class DeviceState:
         return (self.w, self.w_loc[i], self.w_dev[i])[view]
 
     def bytes(self) -> int:
-        return (2 + 3 * self.K) * self.n * 4
+        return (2 + len(self.w_loc) + len(self.pre) + len(self.w_dev)) * self.n * 4

@@ -1,0 +1,180 @@
+"""Bandwidth sweep of the three update kernels on a flat parameter buffer.
+
+    python -m paper_2012_05396_b200.sweep --log2n 16 20 24 26 28 --K 1 4 16 32 --dtype f32 bf16
+
+For every point it times, with CUDA events on the launching stream (3 warm-up + `--reps` timed
+launches, median and minimum reported):
+    sync    ssd_server_sync_update               K*sg + 16 bytes per parameter
+    glu     ssd_worker_glu_update, plain flags   sg + 12 bytes per parameter and worker
+    step    ssd_step in the steps-delay stage    K*(sg+12) + 16 (+4K on refresh, +4K on pull)
+and prints one JSON object per point.  State and gradients are uniform(-1,1) from the seeded
+generators.  Points whose footprint is below four times the L2 size are marked "l2": they are not
+HBM measurements.  Points that do not fit in free device memory are reported as skipped.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import statistics
+import sys
+
+import torch
+
+from . import binding as B
+from . import build as libbuild
+from . import synth
+from .state import DeviceState
+
+L2_BYTES = 126e6
+
+
+def time_launches(fn, reps: int, warmup: int = 3):
+    stream = torch.cuda.current_stream()
+    for _ in range(warmup):
+        fn()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
+    torch.cuda.synchronize()
+    ev[0].record(stream)
+    for r in range(reps):
+        fn()
+        ev[r + 1].record(stream)
+    torch.cuda.synchronize()
+    ms = [ev[r].elapsed_time(ev[r + 1]) for r in range(reps)]
+    return statistics.median(ms), min(ms)
+
+
+def _grads(n, K, dtype):
+    out = []
+    for i in range(K):
+        g = synth.uniform_buffer(synth.STREAM_GRAD, n, worker=i, device="cuda")
+        g.mul_(1e-3)                     # keeps the state bounded over many repetitions
+        out.append(synth.to_bf16(g) if dtype == "bf16" else g)
+    return out
+
+
+def _hp(K, k, dtype):
+    nan = float("nan")
+    return B.make_hparams(K, 0.1, 0.9, 0, k, lr_local=nan, alpha=nan, beta=nan, rescale=nan,
+                          grad_dtype=B.SSD_BF16 if dtype == "bf16" else B.SSD_F32)
+
+
+def _fits(nbytes):
+    free, _ = torch.cuda.mem_get_info()
+    return nbytes * 1.03 + (1 << 30) <= free
+
+
+def point(log2n: int, K: int, dtype: str, kernels, reps: int, peak: float, threads: int, bps: int,
+          vw: int = 0, batch: int = 0):
+    n = 1 << log2n
+    sg = 2 if dtype == "bf16" else 4
+    out = []
+
+    def emit(kernel, footprint, bytes_per_launch, med, mn):
+        gbs = bytes_per_launch / (med * 1e-3) / 1e9
+        out.append({"log2n": log2n, "K": K, "grad_dtype": dtype, "kernel": kernel,
+                    "footprint_bytes": footprint, "l2": footprint < 4 * L2_BYTES,
+                    "bytes_per_launch": bytes_per_launch, "ms_median": med, "ms_min": mn, "gbs": gbs,
+                    "gbs_best": bytes_per_launch / (mn * 1e-3) / 1e9, "frac_of_8TBs": gbs / 8000.0,
+                    "frac_of_measured": gbs / peak, "params_per_s": n / (med * 1e-3)})
+
+    def skip(kernel, footprint):
+        out.append({"log2n": log2n, "K": K, "grad_dtype": dtype, "kernel": kernel,
+                    "footprint_bytes": footprint, "skipped": "does not fit in free device memory"})
+
+    def tune(st):
+        if threads or bps:
+            st.ctx.ssd_set_launch(threads, bps)
+        if vw or batch:
+            st.ctx.ssd_set_kernel_shape(vw, batch)
+
+    w0 = synth.uniform_buffer(synth.STREAM_WEIGHT, n, device="cuda")
+    if "sync" in kernels:
+        # the server alone: a context without a delay stage needs no worker state
+        fp = 2 * n * 4 + K * n * sg
+        if _fits(fp):
+            st = DeviceState([n], _hp(K, 0, dtype), w0, worker_state=False)
+            tune(st)
+            grads = _grads(n, K, dtype)
+            med, mn = time_launches(lambda: st.ctx.ssd_server_sync_update(grads), reps)
+            emit("sync", fp, (K * sg + 16) * n, med, mn)
+            del st, grads
+        else:
+            skip("sync", fp)
+    if "glu" in kernels:
+        # one launch updates one worker, so the worker count does not enter; rotate over up to
+        # four workers' buffers so that consecutive launches touch different memory
+        Kg = min(K, 4)
+        fp = (2 + 3 * Kg) * n * 4 + Kg * n * sg
+        if _fits(fp):
+            st = DeviceState([n], _hp(Kg, 4, dtype), w0, fill=0.0)
+            tune(st)
+            grads = _grads(n, Kg, dtype)
+            for i in range(Kg):
+                st.pre[i].copy_(st.w_loc[i])
+            state = {"i": 0}
+
+            def glu():
+                i = state["i"]
+                st.ctx.ssd_worker_glu_update(i, grads[i], 0)
+                state["i"] = (i + 1) % Kg
+            med, mn = time_launches(glu, reps)
+            emit("glu", fp, (sg + 12) * n, med, mn)
+            del st, grads
+        else:
+            skip("glu", fp)
+    if "step" in kernels:
+        fp = (2 + 3 * K) * n * 4 + K * n * sg
+        if _fits(fp):
+            st = DeviceState([n], _hp(K, 4, dtype), w0, fill=0.0)
+            tune(st)
+            grads = _grads(n, K, dtype)
+            st.ctx.ssd_step(grads)                                   # first GLU call
+            stream = torch.cuda.current_stream()
+            per_flag = {}
+            for _ in range(4):
+                st.ctx.ssd_step(grads)
+            for _ in range(max(reps, 8)):
+                flags = st.ctx.ssd_get_counters()[3]
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                st.ctx.ssd_step(grads)
+                e1.record(stream)
+                torch.cuda.synchronize()
+                per_flag.setdefault(flags, []).append(e0.elapsed_time(e1))
+            for flags, ms in sorted(per_flag.items()):
+                b = K * (sg + 12) + 16 + (4 * K if flags & 2 else 0) + (4 * K if flags & 4 else 0)
+                name = "step" + ("+refresh" if flags & 2 else "") + ("+pull" if flags & 4 else "")
+                emit(name, fp, b * n, statistics.median(ms), min(ms))
+            del st, grads
+        else:
+            skip("step", fp)
+    torch.cuda.empty_cache()
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--log2n", type=int, nargs="+", default=[16, 18, 20, 22, 24, 26, 28])
+    ap.add_argument("--K", type=int, nargs="+", default=[1, 4, 16, 32])
+    ap.add_argument("--dtype", nargs="+", default=["f32", "bf16"], choices=["f32", "bf16"])
+    ap.add_argument("--kernels", nargs="+", default=["sync", "glu", "step"], choices=["sync", "glu", "step"])
+    ap.add_argument("--reps", type=int, default=20)
+    ap.add_argument("--peak", type=float, default=6547.5, help="measured HBM copy rate in GB/s")
+    ap.add_argument("--threads", type=int, default=0)
+    ap.add_argument("--blocks-per-sm", type=int, default=0)
+    ap.add_argument("--vector-elems", type=int, default=0, choices=[0, 4, 8])
+    ap.add_argument("--batch", type=int, default=0, choices=[0, 1, 2, 4, 8])
+    args = ap.parse_args()
+    if not torch.cuda.is_available():
+        raise SystemExit("the sweep needs a CUDA device")
+    libbuild.build_library()
+    for log2n in args.log2n:
+        for K in args.K:
+            for dtype in args.dtype:
+                for rec in point(log2n, K, dtype, args.kernels, args.reps, args.peak, args.threads,
+                                 args.blocks_per_sm, args.vector_elems, args.batch):
+                    print(json.dumps(rec), flush=True)
+
+
+if __name__ == "__main__":
+    main()

@@ -111,7 +111,8 @@ def test_server_alone_is_synchronous_sgd():
     lay = synth.get_layout("resnet20")
     ohp, chp = make_hp(4, 0.1, 0.9, 3, 0, wd=1e-4)
     w0 = synth.init_weights(lay)
-    a, b = DeviceState(lay.numels, chp, w0), DeviceState(lay.numels, chp, w0)
+    a = DeviceState(lay.numels, chp, w0)
+    b = DeviceState(lay.numels, chp, w0, worker_state=False)      # server state only
     ref = oracle.State(ohp, w0.numpy())
     for n in range(6):
         grads = [synth.gradient(lay, n, i, 1e-2, device="cuda") for i in range(4)]
@@ -123,6 +124,9 @@ def test_server_alone_is_synchronous_sgd():
     assert_same(b.w, ref.w, "server-only w")
     assert_same(b.mom, ref.mom, "server-only mom")
     assert b.ctx.ssd_get_counters()[0] == 0
+    with pytest.raises(B.SsdError) as e:
+        b.ctx.ssd_broadcast_weights()
+    assert e.value.status == B.SSD_ERR_STATE
 
 
 def test_glu_update_flags_one_by_one():
@@ -217,3 +221,56 @@ def test_step_host_moves_gradients_and_returns_weights():
         assert_same(w_out, ref.w, f"host w iter {n}")
     compare_states(dev, ref, "step_host")
     assert dev.ctx.ssd_kernel_launches() == 4
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_every_kernel_shape_and_alignment_gives_the_same_bits(bf16):
+    # 256-bit and 128-bit access paths, every load batch, a length with n % 8 == 4, and buffers that
+    # are only 16-byte aligned (which must fall back to 128-bit accesses on their own)
+    K, W, k, iters = 5, 1, 2, 6
+    n = 8 * 1031 + 4
+    ohp, chp = make_hp(K, 0.1, 0.9, W, k, wd=0.01, bf16=bf16)
+    lay = synth.flat(n)
+    w0 = synth.init_weights(lay)
+    grads = [[synth.gradient(lay, it, i, 0.05, device="cuda") for i in range(K)] for it in range(iters)]
+    if bf16:
+        grads = [[synth.to_bf16(g) for g in gs] for gs in grads]
+    ref = oracle.State(ohp, w0.numpy())
+    for gs in grads:
+        ref.step([oracle_grad(g, bf16) for g in gs])
+
+    def offset_copy(t, elems):
+        """A copy of t that starts `elems` elements into a fresh allocation (16-byte aligned only)."""
+        buf = torch.empty(t.numel() + 16, dtype=t.dtype, device="cuda")
+        view = buf[elems:elems + t.numel()]
+        view.copy_(t)
+        assert view.data_ptr() % 32 == 16 and view.data_ptr() % 16 == 0
+        return view
+
+    for vw, batch in [(0, 0), (8, 1), (8, 2), (8, 4), (8, 8), (4, 1), (4, 2), (4, 4), (4, 8)]:
+        for mode in ("fused", "split"):
+            dev = DeviceState(lay.numels, chp, w0)
+            dev.ctx.ssd_set_kernel_shape(vw, batch)
+            for gs in grads:
+                gpu_iteration(dev, gs, mode)
+            torch.cuda.synchronize()
+            compare_states(dev, ref, f"shape vw={vw} batch={batch} {mode}")
+    # misaligned gradient buffers (float32 only matters) and misaligned state
+    shift = 8 if bf16 else 4
+    dev = DeviceState(lay.numels, chp, w0)
+    for gs in grads:
+        gpu_iteration(dev, [offset_copy(g, shift) for g in gs], "fused")
+    torch.cuda.synchronize()
+    compare_states(dev, ref, "misaligned gradients")
+    dev = DeviceState(lay.numels, chp, w0)
+    state = DeviceState.__new__(DeviceState)
+    state.numels, state.n, state.K, state.device = dev.numels, dev.n, K, dev.device
+    state.w, state.mom = offset_copy(dev.w, 4), offset_copy(dev.mom, 4)
+    state.w_loc = [offset_copy(t, 4) for t in dev.w_loc]
+    state.pre = [offset_copy(t, 4) for t in dev.pre]
+    state.w_dev = [offset_copy(t, 4) for t in dev.w_dev]
+    state.ctx = B.Context(lay.numels, chp, state.w, state.mom, state.w_loc, state.pre, state.w_dev)
+    for gs in grads:
+        gpu_iteration(state, gs, "fused")
+    torch.cuda.synchronize()
+    compare_states(state, ref, "misaligned state")
