@@ -43,9 +43,12 @@ WORKLOADS = {
 }
 DEFAULT_WORKLOAD = "vgg16_K16"
 
-# DRAM bytes per launch of step_kernel from an ncu capture (dram__bytes_read.sum +
-# dram__bytes_write.sum), valid only for the kernel sources with this digest.
-NCU_TRAFFIC = {"digest": None, "workload": None, "bytes_per_launch": None}
+# DRAM bytes per parameter of one step_kernel launch (dram__bytes_read.sum + dram__bytes_write.sum
+# from an ncu capture on a flat arena of 2^24 parameters with the same worker count, gradient type
+# and launch shape; the kernel streams, so traffic grows in proportion to N), by iteration flags.
+# Valid only for the kernel sources with this digest.
+NCU_TRAFFIC = {"digest": "53dc9cc50d92e453", "K": 16, "grad_dtype": "f32",
+               "bytes_per_param": {0: 269.98, 2: 332.63, 4: 332.85}}
 
 
 def kernel_digest() -> str:
@@ -295,8 +298,10 @@ def main():
     peak, peak_kind = measured_peak()
     achieved = (sum(bytes_per_launch) / len(bytes_per_launch)) / (statistics.mean(per_launch_ms) * 1e-3) / 1e9
     traffic = None
-    if NCU_TRAFFIC["digest"] == kernel_digest() and NCU_TRAFFIC["workload"] == wl_name:
-        traffic = NCU_TRAFFIC["bytes_per_launch"]
+    if NCU_TRAFFIC["digest"] == kernel_digest() and NCU_TRAFFIC["K"] == K and sg == 4:
+        per = NCU_TRAFFIC["bytes_per_param"]
+        if all((f & 6) in per for f in flags_of):
+            traffic = N * statistics.mean(per[f & 6] for f in flags_of)
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
