@@ -54,25 +54,31 @@ _libs = {}
 def _lib(double: bool):
     if double not in _libs:
         build()
-        lib = C.CDLL(os.path.join(_BUILD, "libssd_oracle_f64.so" if double else "libssd_oracle_f32.so"))
-        lib.oracle_sync_scale.restype = C.c_double if double else C.c_float
-        lib.oracle_sync_scale.argtypes = [C.POINTER(_HP)]
-        lib.oracle_schedule.restype = None
-        lib.oracle_schedule.argtypes = [C.c_int64, C.c_int64, C.c_int64,
-                                        C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
-        lib.oracle_server_update.restype = None
-        lib.oracle_server_update.argtypes = [C.c_int64, C.POINTER(_HP), C.POINTER(C.c_void_p),
-                                             C.c_void_p, C.c_void_p]
-        lib.oracle_glu_update.restype = None
-        lib.oracle_glu_update.argtypes = [C.c_int64, C.POINTER(_HP), C.c_void_p, C.c_void_p,
-                                          C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32]
-        lib.oracle_step.restype = C.c_int32
-        lib.oracle_step.argtypes = [C.POINTER(_State), C.POINTER(_HP), C.POINTER(C.c_void_p),
-                                    C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
-        lib.oracle_real_bytes.restype = C.c_int32
-        assert lib.oracle_real_bytes() == (8 if double else 4)
-        _libs[double] = lib
+        _libs[double] = bind(os.path.join(_BUILD, "libssd_oracle_f64.so" if double else "libssd_oracle_f32.so"),
+                             double)
     return _libs[double]
+
+
+def bind(path: str, double: bool):
+    """Loads one build of ssd_oracle.c and declares its signatures."""
+    lib = C.CDLL(path)
+    lib.oracle_sync_scale.restype = C.c_double if double else C.c_float
+    lib.oracle_sync_scale.argtypes = [C.POINTER(_HP)]
+    lib.oracle_schedule.restype = None
+    lib.oracle_schedule.argtypes = [C.c_int64, C.c_int64, C.c_int64,
+                                    C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+    lib.oracle_server_update.restype = None
+    lib.oracle_server_update.argtypes = [C.c_int64, C.POINTER(_HP), C.POINTER(C.c_void_p),
+                                         C.c_void_p, C.c_void_p]
+    lib.oracle_glu_update.restype = None
+    lib.oracle_glu_update.argtypes = [C.c_int64, C.POINTER(_HP), C.c_void_p, C.c_void_p,
+                                      C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32]
+    lib.oracle_step.restype = C.c_int32
+    lib.oracle_step.argtypes = [C.POINTER(_State), C.POINTER(_HP), C.POINTER(C.c_void_p),
+                                C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+    lib.oracle_real_bytes.restype = C.c_int32
+    assert lib.oracle_real_bytes() == (8 if double else 4)
+    return lib
 
 
 def _ptr(a: np.ndarray) -> int:
