@@ -144,6 +144,21 @@ def dist_setup(n_gpus: int):
     return world, rank, local
 
 
+def max_over_ranks(value: float, device, world: int) -> float:
+    """The slowest rank's time: every rank gets the maximum (identity for a single rank)."""
+    if world <= 1:
+        return float(value)
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(units_per_rank: float, world: int, ms_max: float) -> float:
+    """Units all replicas processed per second, over the slowest rank's time."""
+    return units_per_rank * world / (ms_max * 1e-3)
+
+
 def oracle_sample_run(wl, n_sample: int, steps: int, grads_host, w0_host):
     """Times the CPU oracle, as it stands, on the first n_sample arena elements for `steps`
     delay-stage iterations.  Returns (seconds, bytes moved, params updated, threads used)."""
@@ -288,13 +303,9 @@ def main():
 
     total_ms = ev[0].elapsed_time(ev[-1])
     per_launch_ms = [ev[n].elapsed_time(ev[n + 1]) for n in range(args.steps)]
-    if world > 1:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=dev_name)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, dev_name, world)
     bytes_per_launch = [step_bytes_per_param(K, sg, f) * N for f in flags_of]
-    total_bytes = float(sum(bytes_per_launch)) * world
-    value = total_bytes / (total_ms * 1e-3) / 1e9
+    value = whole_job_rate(float(sum(bytes_per_launch)), world, total_ms) / 1e9
     peak, peak_kind = measured_peak()
     achieved = (sum(bytes_per_launch) / len(bytes_per_launch)) / (statistics.mean(per_launch_ms) * 1e-3) / 1e9
     traffic = None
@@ -307,7 +318,7 @@ def main():
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "params_per_s": N * args.steps * world / (total_ms * 1e-3),
+        "params_per_s": whole_job_rate(float(N) * args.steps, world, total_ms),
         "frac_of_nominal_8TBs": value / world / NOMINAL_HBM_GBS,
         "wall_ms_per_step": t_wall / args.steps * 1e3,
         "config": {"workload": wl_name, "layout": wl["layout"], "params": lay.numel, "tensors": lay.num_tensors,
@@ -346,12 +357,9 @@ def main():
         e1.record(stream)
         torch.cuda.synchronize()
         e_ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([e_ms], dtype=torch.float64, device=dev_name)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e_ms = float(t.item())
-        e_bytes = float(sum(step_bytes_per_param(K, sg, f) * N for f in e_flags)) * world
-        e2e = {"value": e_bytes / (e_ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": K * N * sg,
+        e_ms = max_over_ranks(e_ms, dev_name, world)
+        e_bytes = float(sum(step_bytes_per_param(K, sg, f) * N for f in e_flags))
+        e2e = {"value": whole_job_rate(e_bytes, world, e_ms) / 1e9, "unit": UNIT, "h2d_bytes_per_step": K * N * sg,
                "d2h_bytes_per_step": N * 4, "steps": args.e2e_steps, "ms_per_step": e_ms / args.e2e_steps,
                "call": "ssd_step_host"}
         del host_grads, host_w
