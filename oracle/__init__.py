@@ -39,7 +39,8 @@ class _HP(C.Structure):
     _fields_ = [("K", C.c_int32), ("grad_bf16", C.c_int32), ("W", C.c_int64), ("k", C.c_int64),
                 ("lr", C.c_float), ("m", C.c_float), ("wd", C.c_float),
                 ("lr_loc", C.c_float), ("alpha", C.c_float), ("beta", C.c_float),
-                ("rescale", C.c_float)]
+                ("rescale", C.c_float), ("T", C.c_int32), ("tensor_end", C.c_void_p),
+                ("lr_mult", C.c_void_p), ("wd_mult", C.c_void_p), ("arena_index", C.c_void_p)]
 
 
 class _State(C.Structure):
@@ -104,11 +105,24 @@ class Hyper:
         self.alpha, self.beta = f32(alpha), f32(beta)
         self.rescale = f32(1.0 / K) if rescale is None else f32(rescale)
         self.grad_bf16 = bool(grad_bf16)
+        self.tensor_end = self.lr_mult = self.wd_mult = self.arena_index = None
+
+    def set_tensor_scales(self, tensor_end, lr_mult, wd_mult, arena_index=None) -> None:
+        """Per-tensor multipliers: tensor t covers arena positions up to tensor_end[t] (exclusive,
+        padding included).  arena_index maps local elements to arena positions for sampled runs."""
+        self.tensor_end = np.ascontiguousarray(tensor_end, dtype=np.int64)
+        self.lr_mult = np.ascontiguousarray(lr_mult, dtype=np.float32)
+        self.wd_mult = np.ascontiguousarray(wd_mult, dtype=np.float32)
+        assert self.tensor_end.shape == self.lr_mult.shape == self.wd_mult.shape
+        self.arena_index = None if arena_index is None else np.ascontiguousarray(arena_index, dtype=np.int64)
 
     def c_struct(self) -> _HP:
+        T = 0 if self.tensor_end is None else len(self.tensor_end)
+        ptr = lambda a: None if a is None else a.ctypes.data
         return _HP(self.K, int(self.grad_bf16), self.W, self.k, float(self.lr), float(self.m),
                    float(self.wd), float(self.lr_loc), float(self.alpha), float(self.beta),
-                   float(self.rescale))
+                   float(self.rescale), T, ptr(self.tensor_end), ptr(self.lr_mult), ptr(self.wd_mult),
+                   ptr(self.arena_index))
 
 
 def schedule(n: int, W: int, k: int):

@@ -44,6 +44,15 @@ typedef struct {
     float lr, m, wd;      /* server: learning rate, momentum, weight decay       */
     float lr_loc, alpha, beta;   /* GLU: local lr and the two mixing coefficients */
     float rescale;        /* factor applied to the K-sum (1/K = average)         */
+    /* Optional per-tensor multipliers (the paper uses one lr and one wd for the whole
+     * model; per-tensor values are the usual refinement, e.g. no decay on BN and bias).
+     * T == 0: uniform.  Tensor t covers arena positions [tensor_end[t-1], tensor_end[t]). */
+    int32_t T;
+    const int64_t *tensor_end;   /* T increasing exclusive end positions             */
+    const float *lr_mult;        /* multiplies lr and lr_loc of tensor t             */
+    const float *wd_mult;        /* multiplies wd of tensor t                        */
+    const int64_t *arena_index;  /* optional: arena position of local element j (for
+                                    runs on a gathered sample of the arena)          */
 } oracle_hp;
 
 typedef struct {
@@ -73,10 +82,36 @@ static real grad_at(const void *g, int bf16, int64_t j)
 
 /* grad_sync scale (1-m)/(lr*k) of Section 3.3, from the float-typed
  * hyper-parameters, evaluated in double and rounded once to `real`. */
-real oracle_sync_scale(const oracle_hp *hp)
+static real sync_scale_for(float lr, float m, int64_t k)
 {
-    if (hp->k <= 0) return (real)0;
-    return (real)((1.0 - (double)hp->m) / ((double)hp->lr * (double)hp->k));
+    if (k <= 0) return (real)0;
+    return (real)((1.0 - (double)m) / ((double)lr * (double)k));
+}
+
+real oracle_sync_scale(const oracle_hp *hp) { return sync_scale_for(hp->lr, hp->m, hp->k); }
+
+/* The four scalars that may differ per tensor, for local element j.  With
+ * multipliers, tensor t uses lr*lr_mult[t], lr_loc*lr_mult[t], wd*wd_mult[t]
+ * (each one float multiplication) and the grad_sync scale of its own lr. */
+typedef struct { real lr, wd, lr_loc, c; } tensor_scalars;
+
+static tensor_scalars scalars_at(const oracle_hp *hp, int64_t j)
+{
+    tensor_scalars s;
+    if (hp->T == 0) {
+        s.lr = (real)hp->lr; s.wd = (real)hp->wd; s.lr_loc = (real)hp->lr_loc;
+        s.c = sync_scale_for(hp->lr, hp->m, hp->k);
+        return s;
+    }
+    int64_t pos = hp->arena_index ? hp->arena_index[j] : j;
+    int32_t t = 0;
+    while (t < hp->T - 1 && pos >= hp->tensor_end[t]) ++t;
+    float lr_t = hp->lr * hp->lr_mult[t];
+    float wd_t = hp->wd * hp->wd_mult[t];
+    float lr_loc_t = hp->lr_loc * hp->lr_mult[t];
+    s.lr = (real)lr_t; s.wd = (real)wd_t; s.lr_loc = (real)lr_loc_t;
+    s.c = sync_scale_for(lr_t, hp->m, hp->k);
+    return s;
 }
 
 /* Stage and event flags of 0-based iteration n (Algorithm 1 and Algorithm 2).
@@ -106,9 +141,12 @@ void oracle_schedule(int64_t n, int64_t W, int64_t k, int32_t *stage, int32_t *f
 void oracle_server_update(int64_t N, const oracle_hp *hp, const void *const *g,
                           real *w, real *mom)
 {
-    const real lr = (real)hp->lr, m = (real)hp->m, wd = (real)hp->wd;
+    const real m = (real)hp->m;
     const real rescale = (real)hp->rescale;
+    const tensor_scalars uniform = scalars_at(hp, 0);
     for (int64_t j = 0; j < N; ++j) {
+        const tensor_scalars ts = hp->T ? scalars_at(hp, j) : uniform;
+        const real lr = ts.lr, wd = ts.wd;
         real s = grad_at(g[0], hp->grad_bf16, j);
         for (int32_t i = 1; i < hp->K; ++i)
             s = s + grad_at(g[i], hp->grad_bf16, j);
@@ -134,10 +172,11 @@ void oracle_glu_update(int64_t N, const oracle_hp *hp, const void *g,
                        real *w_loc, real *pre, real *w_dev, const real *w_server,
                        int32_t flags)
 {
-    const real lr_loc = (real)hp->lr_loc, alpha = (real)hp->alpha, beta = (real)hp->beta;
-    const real wd = (real)hp->wd;
-    const real c = oracle_sync_scale(hp);
+    const real alpha = (real)hp->alpha, beta = (real)hp->beta;
+    const tensor_scalars uniform = scalars_at(hp, 0);
     for (int64_t j = 0; j < N; ++j) {
+        const tensor_scalars ts = hp->T ? scalars_at(hp, j) : uniform;
+        const real lr_loc = ts.lr_loc, wd = ts.wd, c = ts.c;
         if (flags & F_FIRST) pre[j] = w_loc[j];
         real diff = pre[j] - w_loc[j];
         real grad_sync = diff * c;

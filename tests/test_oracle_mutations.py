@@ -12,7 +12,7 @@ import pytest
 
 import oracle
 from tests import golden_trace
-from tests.test_oracle_pins import paper_counters
+from tests.test_oracle_pins import paper_counters, per_tensor_composition_holds
 
 SRC = os.path.join(os.path.dirname(oracle.__file__), "ssd_oracle.c")
 
@@ -32,14 +32,18 @@ MUTATIONS = [
      "if (flags & F_REFRESH) pre[j] = w_loc[j];\n        real diff = pre[j] - w_loc[j];\n        real grad_sync = diff * c;"),
     ("refresh stores the updated weight", "if (flags & F_REFRESH) pre[j] = w_loc[j];\n        real local", "real local"),
     ("pull hands the global weight to the devices", "w_dev[j] = w_loc[j];\n            w_loc[j] = w_server[j];", "w_loc[j] = w_server[j];\n            w_dev[j] = w_loc[j];"),
-    ("scale uses lr_loc", "((double)hp->lr * (double)hp->k)", "((double)hp->lr_loc * (double)hp->k)"),
-    ("scale forgets k", "((double)hp->lr * (double)hp->k)", "((double)hp->lr)"),
+    ("scale uses lr_loc", "s.c = sync_scale_for(hp->lr, hp->m, hp->k);", "s.c = sync_scale_for(hp->lr_loc, hp->m, hp->k);"),
+    ("scale forgets k", "((double)lr * (double)k)", "((double)lr)"),
     ("workers use worker 0's gradient", "oracle_glu_update(st->N, hp, g[i],", "oracle_glu_update(st->N, hp, g[0],"),
     ("server runs after the workers", None, None),       # handled below: moves the call
     ("warm-up one iteration short", "n == W - 1) ? F_COPY", "n == W - 2) ? F_COPY"),
     ("pull one iteration early", "d % k == k - 1", "(d + 1) % k == k - 1"),
     ("refresh on the first call", "if (d > 0 && d % k == 0)", "if (d % k == 0)"),
     ("warm-up off by one", "if (k == 0 || n < W)", "if (k == 0 || n <= W)"),
+    ("tensor lookup off by one", "pos >= hp->tensor_end[t]", "pos > hp->tensor_end[t]"),
+    ("local lr ignores the tensor's multiplier", "float lr_loc_t = hp->lr_loc * hp->lr_mult[t];", "float lr_loc_t = hp->lr_loc;"),
+    ("decay multiplier taken from lr_mult", "float wd_t = hp->wd * hp->wd_mult[t];", "float wd_t = hp->wd * hp->lr_mult[t];"),
+    ("per-tensor scale from the global lr", "s.c = sync_scale_for(lr_t, hp->m, hp->k);", "s.c = sync_scale_for(hp->lr, hp->m, hp->k);"),
 ]
 
 
@@ -86,7 +90,7 @@ def traces_pass(lib):
                 ref = paper_counters(W, k, W + 3 * k + 2)
                 if [oracle.schedule(n, W, k) for n in range(len(ref))] != ref:
                     return False
-        return True
+        return per_tensor_composition_holds()
     finally:
         if saved is not None:
             oracle._libs[False] = saved

@@ -461,3 +461,93 @@ def test_float32_tracks_double_shadow():
     np.testing.assert_allclose(a.w, b.w, rtol=1e-5, atol=1e-6)
     for i in range(K):
         np.testing.assert_allclose(a.w_loc[i], b.w_loc[i], rtol=1e-4, atol=1e-5)
+
+
+# ---------------------------------------------------------------------------
+# per-tensor multipliers: they must reduce to uniform runs on each tensor's slice
+# ---------------------------------------------------------------------------
+
+def per_tensor_composition_holds():
+    """A run with per-tensor multipliers equals, tensor by tensor (padding included), a uniform run
+    whose lr, lr_loc and wd are the tensor's products.  Returns False on the first mismatch."""
+    rng = np.random.default_rng(11)
+    K, W, k, T = 3, 2, 2, 9
+    ends = np.array([8, 12, 24], np.int64)           # tensors of 5, 1 and 10 elements, padded to 4s
+    lr_mult = np.array([1.0, 0.5, 2.0], f32)
+    wd_mult = np.array([1.0, 0.0, 3.0], f32)
+    N = int(ends[-1])
+    w0 = rng.standard_normal(N).astype(f32)
+    stream = [rng_grads(rng, K, N, 0.1) for _ in range(T)]
+    hp = Hyper(K=K, lr=0.1, m=0.9, W=W, k=k, wd=0.01)
+    hp.set_tensor_scales(ends, lr_mult, wd_mult)
+    full = State(hp, w0)
+    for gs in stream:
+        full.step(gs)
+    lo = 0
+    for t, hi in enumerate(ends):
+        hi = int(hi)
+        one = Hyper(K=K, lr=f32(0.1) * lr_mult[t], m=0.9, W=W, k=k, wd=f32(0.01) * wd_mult[t],
+                    lr_loc=hp.lr_loc * lr_mult[t])
+        part = State(one, w0[lo:hi])
+        for gs in stream:
+            part.step([np.ascontiguousarray(g[lo:hi]) for g in gs])
+        same = np.array_equal(full.w[lo:hi], part.w) and np.array_equal(full.mom[lo:hi], part.mom)
+        for i in range(K):
+            same = same and np.array_equal(full.w_loc[i][lo:hi], part.w_loc[i]) \
+                and np.array_equal(full.pre[i][lo:hi], part.pre[i]) \
+                and np.array_equal(full.w_dev[i][lo:hi], part.w_dev[i])
+        if not same:
+            return False
+        lo = hi
+    # a gathered sample of the arena, told where its elements sit, follows the same trajectories
+    idx = np.array([0, 4, 7, 8, 11, 12, 23], np.int64)
+    hs = Hyper(K=K, lr=0.1, m=0.9, W=W, k=k, wd=0.01)
+    hs.set_tensor_scales(ends, lr_mult, wd_mult, arena_index=idx)
+    samp = State(hs, w0[idx])
+    for gs in stream:
+        samp.step([np.ascontiguousarray(g[idx]) for g in gs])
+    return bool(np.array_equal(samp.w, full.w[idx]) and np.array_equal(samp.w_loc[1], full.w_loc[1][idx])
+                and np.array_equal(samp.pre[2], full.pre[2][idx]))
+
+
+def test_per_tensor_multipliers_compose_from_uniform_runs():
+    assert per_tensor_composition_holds()
+
+
+def test_unit_multipliers_equal_the_uniform_path():
+    rng = np.random.default_rng(12)
+    K, N, T = 2, 16, 9
+    w0 = rng.standard_normal(N).astype(f32)
+    stream = [rng_grads(rng, K, N, 0.1) for _ in range(T)]
+    a, _ = run_config(Hyper(K=K, lr=0.1, m=0.9, W=1, k=3, wd=0.01), w0, stream)
+    hp = Hyper(K=K, lr=0.1, m=0.9, W=1, k=3, wd=0.01)
+    hp.set_tensor_scales([4, 16], [1.0, 1.0], [1.0, 1.0])
+    b, _ = run_config(hp, w0, stream)
+    np.testing.assert_array_equal(a.w, b.w)
+    for i in range(K):
+        np.testing.assert_array_equal(a.w_loc[i], b.w_loc[i])
+        np.testing.assert_array_equal(a.pre[i], b.pre[i])
+
+
+def test_server_trajectory_independent_of_schedule_with_multipliers_and_lr_changes():
+    # the server never sees the delay mechanism, also with per-tensor values and an lr schedule
+    rng = np.random.default_rng(13)
+    K, N, T = 2, 12, 15
+    w0 = rng.standard_normal(N).astype(f32)
+    stream = [rng_grads(rng, K, N) for _ in range(T)]
+
+    def run(W, k):
+        hp = Hyper(K=K, lr=0.1, m=0.9, W=W, k=k, wd=0.01)
+        hp.set_tensor_scales([4, 12], [1.0, 0.25], [0.0, 1.0])
+        st = State(hp, w0)
+        for n, gs in enumerate(stream):
+            if n == 6:
+                hp.lr = f32(0.05)                     # a step of the learning-rate schedule
+                hp.lr_loc = f32(0.2)
+            st.step(gs)
+        return st
+    ref = run(0, 0)
+    for W, k in ((2, 4), (3, 1), (0, 2)):
+        st = run(W, k)
+        np.testing.assert_array_equal(st.w, ref.w)
+        np.testing.assert_array_equal(st.mom, ref.mom)
