@@ -223,6 +223,8 @@ def main():
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--per-tensor", action="store_true",
+                    help="per-tensor hyper-parameters: weight decay 5e-4 on conv/FC weights only")
     ap.add_argument("--threads", type=int, default=0, help="threads per block (0 = library default)")
     ap.add_argument("--blocks-per-sm", type=int, default=0, help="resident blocks per SM (0 = default)")
     args = ap.parse_args()
@@ -260,10 +262,13 @@ def main():
         raise SystemExit(f"workload needs {need / 2**30:.1f} GiB, only {free / 2**30:.1f} GiB free")
 
     nan = float("nan")
-    hp = B.make_hparams(K, wl["lr"], wl["m"], wl["W"], wl["k"], lr_local=nan, alpha=nan, beta=nan,
-                        rescale=nan, grad_dtype=B.SSD_F32)
+    hp = B.make_hparams(K, wl["lr"], wl["m"], wl["W"], wl["k"], wd=5e-4 if args.per_tensor else 0.0,
+                        lr_local=nan, alpha=nan, beta=nan, rescale=nan, grad_dtype=B.SSD_F32)
     w0 = synth.init_weights(lay, device=dev_name)
     st = DeviceState(lay.numels, hp, w0, device=dev_name, fill=0.0)
+    if args.per_tensor:
+        table = torch.empty(st.ctx.ssd_tensor_table_bytes(), dtype=torch.uint8, device=dev_name)
+        st.ctx.ssd_set_tensor_scales(None, [1.0 if kind == "he" else 0.0 for kind in lay.kinds], table)
     if args.threads or args.blocks_per_sm:
         st.ctx.ssd_set_launch(args.threads, args.blocks_per_sm)
     mask = synth.valid_mask(lay, dev_name) if N != lay.numel else None
@@ -324,6 +329,7 @@ def main():
         "config": {"workload": wl_name, "layout": wl["layout"], "params": lay.numel, "tensors": lay.num_tensors,
                    "workers": K, "delay_k": wl["k"], "ssd_warmup_iters": wl["W"], "grad_dtype": "f32",
                    "stage": "steps-delay", "kernel": "fused ssd_step", "replicas": world,
+                   "hyper_parameters": "per tensor" if args.per_tensor else "uniform",
                    "device_bytes": st.bytes() + n_sets * K * N * sg,
                    "l2": "inputs larger than L2 (no flush needed)"
                    if st.bytes() > 4 * 126e6 else "L2-resident: not an HBM measurement"},

@@ -225,8 +225,26 @@ ssd_status ssd_set_counters(ssd_ctx *ctx, int64_t iter, int64_t loc_update);
 
 /* Changes the learning rates between iterations and re-derives c.  NaN keeps a
  * value.  (The geometric-series argument behind grad_sync assumes a constant lr;
- * after a change grad_sync is an estimate under the new lr.) */
-ssd_status ssd_set_lr(ssd_ctx *ctx, float lr, float lr_local);
+ * after a change grad_sync is an estimate under the new lr.)  When per-tensor
+ * scales are set, the table is rebuilt and its upload enqueued on `cuda_stream`,
+ * so the change is ordered with the steps enqueued on that stream. */
+ssd_status ssd_set_lr(ssd_ctx *ctx, float lr, float lr_local, void *cuda_stream);
+
+/* Per-tensor hyper-parameters.  The paper uses one lr and one wd for the whole
+ * model; this is the usual refinement (e.g. no weight decay on BN and bias).
+ * Tensor t, padding up to the next tensor included, then uses
+ *     lr_t = lr * lr_mult[t],  lr_local_t = lr_local * lr_mult[t],  wd_t = wd * wd_mult[t]
+ * (one float multiplication each) and c_t = (1 - m) / (lr_t * k), in place of the
+ * uniform values, in the server rule and in the GLU rule alike.
+ * lr_mult, wd_mult: HOST arrays of num_tensors floats (NULL = all 1; lr_mult > 0).
+ * device_table: caller-owned DEVICE memory of ssd_tensor_table_bytes() bytes,
+ * 16-byte aligned, which the kernels read from then on and which must stay
+ * valid until it is replaced; the library fills it by a copy enqueued on
+ * `cuda_stream`.  device_table == NULL returns to uniform hyper-parameters.
+ * Errors: SSD_ERR_ARG, SSD_ERR_ALIGN, SSD_ERR_CUDA. */
+ssd_status ssd_tensor_table_bytes(const ssd_ctx *ctx, int64_t *bytes);
+ssd_status ssd_set_tensor_scales(ssd_ctx *ctx, const float *lr_mult, const float *wd_mult,
+                                 void *device_table, void *cuda_stream);
 
 /* Resolved hyper-parameters as the kernels use them, and the derived c. */
 ssd_status ssd_get_hparams(const ssd_ctx *ctx, ssd_hparams *resolved, float *sync_scale);

@@ -29,7 +29,7 @@ EXPORTS = (
     "ssd_arena_numel", "ssd_init", "ssd_destroy", "ssd_tensor_offset", "ssd_schedule",
     "ssd_server_sync_update", "ssd_worker_glu_update", "ssd_worker_local_step", "ssd_advance",
     "ssd_step", "ssd_step_host", "ssd_broadcast_weights", "ssd_worker_weights", "ssd_get_counters",
-    "ssd_set_counters", "ssd_set_lr", "ssd_get_hparams", "ssd_set_launch", "ssd_set_kernel_shape",
+    "ssd_set_counters", "ssd_set_lr", "ssd_tensor_table_bytes", "ssd_set_tensor_scales", "ssd_get_hparams", "ssd_set_launch", "ssd_set_kernel_shape",
     "ssd_kernel_launches",
     "ssd_status_str", "ssd_last_cuda_error",
 )
@@ -87,7 +87,9 @@ def lib():
             "ssd_worker_weights": (i32, [vp, i32, P(vp), P(i32)]),
             "ssd_get_counters": (i32, [vp, P(i64), P(i64), P(i32), P(i32)]),
             "ssd_set_counters": (i32, [vp, i64, i64]),
-            "ssd_set_lr": (i32, [vp, C.c_float, C.c_float]),
+            "ssd_set_lr": (i32, [vp, C.c_float, C.c_float, vp]),
+            "ssd_tensor_table_bytes": (i32, [vp, P(i64)]),
+            "ssd_set_tensor_scales": (i32, [vp, P(C.c_float), P(C.c_float), vp, vp]),
             "ssd_get_hparams": (i32, [vp, P(ssd_hparams), P(C.c_float)]),
             "ssd_set_launch": (i32, [vp, i32, i32]),
             "ssd_set_kernel_shape": (i32, [vp, i32, i32]),
@@ -227,8 +229,21 @@ class Context:
     def ssd_set_counters(self, it: int, loc_update: int):
         self._check(lib().ssd_set_counters(self._h, it, loc_update), "ssd_set_counters")
 
-    def ssd_set_lr(self, lr: float = math.nan, lr_local: float = math.nan):
-        self._check(lib().ssd_set_lr(self._h, lr, lr_local), "ssd_set_lr")
+    def ssd_set_lr(self, lr: float = math.nan, lr_local: float = math.nan, stream=None):
+        self._check(lib().ssd_set_lr(self._h, lr, lr_local, _stream(stream)), "ssd_set_lr")
+
+    def ssd_tensor_table_bytes(self) -> int:
+        out = C.c_int64()
+        self._check(lib().ssd_tensor_table_bytes(self._h, C.byref(out)), "ssd_tensor_table_bytes")
+        return out.value
+
+    def ssd_set_tensor_scales(self, lr_mult, wd_mult, device_table, stream=None):
+        """lr_mult / wd_mult: sequences of floats or None; device_table: tensor / address / None."""
+        def arr(x):
+            return None if x is None else (C.c_float * len(x))(*[float(v) for v in x])
+        self._table = device_table                       # keep the tensor alive
+        self._check(lib().ssd_set_tensor_scales(self._h, arr(lr_mult), arr(wd_mult), _ptr(device_table),
+                                                _stream(stream)), "ssd_set_tensor_scales")
 
     def ssd_get_hparams(self):
         hp, c = ssd_hparams(), C.c_float()

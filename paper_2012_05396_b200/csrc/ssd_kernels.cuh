@@ -45,6 +45,15 @@ struct Scalars {
     float lr_loc, alpha, beta, c;  // GLU; c = (1-m)/(lr*k)
 };
 
+// Optional per-tensor scalars (device memory, filled by the host): tensor t covers arena
+// positions [end[t-1], end[t]) and uses scal[t] = {lr, wd, lr_loc, c} instead of the uniform
+// values in Scalars.  T == 0: uniform.
+struct TensorTable {
+    const int64_t *end;
+    const float4 *scal;
+    int T;
+};
+
 struct SyncParams {
     const void *g[kMaxWorkers];
     float *w_loc[kMaxWorkers];     // written when flags has kCopy
@@ -52,6 +61,7 @@ struct SyncParams {
     int64_t n;
     int K, flags;
     Scalars s;
+    TensorTable tt;
 };
 
 struct GluParams {
@@ -61,6 +71,7 @@ struct GluParams {
     int64_t n;
     int flags;
     Scalars s;
+    TensorTable tt;
 };
 
 struct StepParams {
@@ -72,6 +83,7 @@ struct StepParams {
     int64_t n;
     int K, flags;
     Scalars s;
+    TensorTable tt;
 };
 
 struct CopyParams {
@@ -200,11 +212,50 @@ __device__ __forceinline__ float glu_elem(float g, float wl, float pre, const Sc
 }
 
 // ---------------------------------------------------------------------------
+// Per-tensor scalars.  Tensors start on multiples of 4 elements, so each group of
+// 4 consecutive elements lies in one tensor; a vector of 8 may straddle two.  The
+// search runs after the thread's loads have been issued, under their latency.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ int tensor_of(const TensorTable &tt, int64_t e)
+{
+    int lo = 0, hi = tt.T - 1;                 // first t with end[t] > e
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (__ldg(tt.end + mid) > e) hi = mid; else lo = mid + 1;
+    }
+    return lo;
+}
+
+__device__ __forceinline__ Scalars with_tensor(Scalars s, const TensorTable &tt, int t)
+{
+    const float4 v = __ldg(tt.scal + t);
+    s.lr = v.x; s.wd = v.y; s.lr_loc = v.z; s.c = v.w;
+    return s;
+}
+
+// Scalars of each 4-element group of the vector at element offset e.
+template <bool PT, int VW> struct GroupScalars {
+    Scalars g[VW / 4];
+    __device__ __forceinline__ GroupScalars(const Scalars &uniform, const TensorTable &tt, int64_t e)
+    {
+#pragma unroll
+        for (int q = 0; q < VW / 4; ++q) g[q] = uniform;
+        if (PT) {
+            const int t = tensor_of(tt, e);
+            g[0] = with_tensor(uniform, tt, t);
+            if (VW == 8)
+                g[VW / 4 - 1] = (e + 4 < __ldg(tt.end + t)) ? g[0] : with_tensor(uniform, tt, tensor_of(tt, e + 4));
+        }
+    }
+    __device__ __forceinline__ const Scalars &at(int l) const { return g[l >> 2]; }
+};
+
+// ---------------------------------------------------------------------------
 // Bodies, written once for a vector of VW elements at element offset e.
 // B = workers whose loads are issued together before any is consumed.
 // ---------------------------------------------------------------------------
 
-template <int GT, int VW, int B>
+template <int GT, int VW, int B, bool PT>
 __device__ __forceinline__ void sync_at(const SyncParams &p, int64_t e)
 {
     Vec<VW> w = ld_f32<VW>(p.w, e);
@@ -224,15 +275,16 @@ __device__ __forceinline__ void sync_at(const SyncParams &p, int64_t e)
             }
         }
     }
+    const GroupScalars<PT, VW> sc(p.s, p.tt, e);
 #pragma unroll
-    for (int l = 0; l < VW; ++l) server_elem(sum.v[l], w.v[l], mom.v[l], p.s);
+    for (int l = 0; l < VW; ++l) server_elem(sum.v[l], w.v[l], mom.v[l], sc.at(l));
     st_f32<VW>(p.mom, e, mom);
     st_f32<VW>(p.w, e, w);
     if (p.flags & kCopy)
         for (int i = 0; i < p.K; ++i) st_f32<VW>(p.w_loc[i], e, w);
 }
 
-template <int GT, int VW>
+template <int GT, int VW, bool PT>
 __device__ __forceinline__ void glu_at(const GluParams &p, int64_t e)
 {
     const bool first = p.flags & kFirst, refresh = p.flags & kRefresh, pull = p.flags & kPull;
@@ -242,8 +294,9 @@ __device__ __forceinline__ void glu_at(const GluParams &p, int64_t e)
     Vec<VW> wg;
     if (pull) wg = ld_f32<VW>(p.w, e);
     Vec<VW> r;
+    const GroupScalars<PT, VW> sc(p.s, p.tt, e);
 #pragma unroll
-    for (int l = 0; l < VW; ++l) r.v[l] = glu_elem(g.get(l), wl.v[l], pr.v[l], p.s);
+    for (int l = 0; l < VW; ++l) r.v[l] = glu_elem(g.get(l), wl.v[l], pr.v[l], sc.at(l));
     if (first || refresh) st_f32<VW>(p.pre, e, wl);
     if (pull) {
         st_f32<VW>(p.w_dev, e, r);
@@ -253,13 +306,14 @@ __device__ __forceinline__ void glu_at(const GluParams &p, int64_t e)
     }
 }
 
-template <int GT, int VW, int B>
+template <int GT, int VW, int B, bool PT>
 __device__ __forceinline__ void step_at(const StepParams &p, int64_t e)
 {
     const bool first = p.flags & kFirst, refresh = p.flags & kRefresh, pull = p.flags & kPull;
     Vec<VW> w = ld_f32<VW>(p.w, e);
     Vec<VW> mom = ld_f32<VW>(p.mom, e);
     Vec<VW> sum;
+    GroupScalars<PT, VW> sc(p.s, p.tt, e);
     for (int i0 = 0; i0 < p.K; i0 += B) {
         Grad<GT, VW> g[B];
         Vec<VW> wl[B], pr[B];
@@ -280,7 +334,7 @@ __device__ __forceinline__ void step_at(const StepParams &p, int64_t e)
                 for (int l = 0; l < VW; ++l) {
                     const float gl = g[b].get(l);
                     sum.v[l] = (i == 0) ? gl : __fadd_rn(sum.v[l], gl);
-                    r.v[l] = glu_elem(gl, wl[b].v[l], first ? wl[b].v[l] : pr[b].v[l], p.s);
+                    r.v[l] = glu_elem(gl, wl[b].v[l], first ? wl[b].v[l] : pr[b].v[l], sc.at(l));
                 }
                 if (first || refresh) st_f32<VW>(p.pre[i], e, wl[b]);
                 st_f32<VW>(pull ? p.w_dev[i] : p.w_loc[i], e, r);
@@ -288,7 +342,7 @@ __device__ __forceinline__ void step_at(const StepParams &p, int64_t e)
         }
     }
 #pragma unroll
-    for (int l = 0; l < VW; ++l) server_elem(sum.v[l], w.v[l], mom.v[l], p.s);
+    for (int l = 0; l < VW; ++l) server_elem(sum.v[l], w.v[l], mom.v[l], sc.at(l));
     st_f32<VW>(p.mom, e, mom);
     st_f32<VW>(p.w, e, w);
     if (pull)
@@ -314,22 +368,23 @@ __device__ __forceinline__ void step_at(const StepParams &p, int64_t e)
         }                                                                                 \
     } while (0)
 
-template <int GT, int VW, int B>
+// PT: per-tensor scalars from the table instead of the uniform ones.
+template <int GT, int VW, int B, bool PT>
 __global__ void __launch_bounds__(kMaxThreads) sync_kernel(const __grid_constant__ SyncParams p)
 {
-    SSD_SWEEP(p.n, VW, (sync_at<GT, VW, B>(p, e)), (sync_at<GT, 4, B>(p, e)));
+    SSD_SWEEP(p.n, VW, (sync_at<GT, VW, B, PT>(p, e)), (sync_at<GT, 4, B, PT>(p, e)));
 }
 
-template <int GT, int VW>
+template <int GT, int VW, bool PT>
 __global__ void __launch_bounds__(kMaxThreads) glu_kernel(const __grid_constant__ GluParams p)
 {
-    SSD_SWEEP(p.n, VW, (glu_at<GT, VW>(p, e)), (glu_at<GT, 4>(p, e)));
+    SSD_SWEEP(p.n, VW, (glu_at<GT, VW, PT>(p, e)), (glu_at<GT, 4, PT>(p, e)));
 }
 
-template <int GT, int VW, int B>
+template <int GT, int VW, int B, bool PT>
 __global__ void __launch_bounds__(kMaxThreads) step_kernel(const __grid_constant__ StepParams p)
 {
-    SSD_SWEEP(p.n, VW, (step_at<GT, VW, B>(p, e)), (step_at<GT, 4, B>(p, e)));
+    SSD_SWEEP(p.n, VW, (step_at<GT, VW, B, PT>(p, e)), (step_at<GT, 4, B, PT>(p, e)));
 }
 
 template <int VW> __device__ __forceinline__ void copy_at(const CopyParams &p, int64_t e)

@@ -36,6 +36,10 @@ struct ssd_ctx {
     bool state32 = false;             // every state buffer is 32-byte aligned
     int threads = 0, blocks_per_sm = 0;     // 0: the kernel's default shape
     int force_vw = 0, force_batch = 0;      // 0: chosen from alignment and K
+    // per-tensor scalars: host copies of the multipliers and the caller's device table
+    std::vector<float> lr_mult, wd_mult;
+    void *tensor_table = nullptr;
+    std::vector<unsigned char> table_image;   // what was last uploaded
     int64_t launches = 0;
     Device dev;
     std::string cuda_error;
@@ -207,6 +211,46 @@ Shape step_shape(const ssd_ctx *c, int flags, bool wide_ok)
 
 Shape glu_shape(const ssd_ctx *c, bool wide_ok) { return finish_shape(c, Shape{8, 1, 256, 0}, wide_ok, 1); }
 
+size_t table_end_bytes(const ssd_ctx *c) { return (c->offsets.size() * sizeof(int64_t) + 15) / 16 * 16; }
+size_t table_bytes(const ssd_ctx *c) { return table_end_bytes(c) + c->offsets.size() * sizeof(float4); }
+
+TensorTable table_of(const ssd_ctx *c)
+{
+    TensorTable tt{};
+    if (c->tensor_table) {
+        tt.end = static_cast<const int64_t *>(c->tensor_table);
+        tt.scal = reinterpret_cast<const float4 *>(static_cast<const unsigned char *>(c->tensor_table) +
+                                                   table_end_bytes(c));
+        tt.T = static_cast<int>(c->offsets.size());
+    }
+    return tt;
+}
+
+// Builds the table image from the current hyper-parameters and multipliers and enqueues its
+// upload.  Tensor t: lr*lr_mult[t], wd*wd_mult[t], lr_local*lr_mult[t] (one float multiplication
+// each) and the grad_sync scale of its own lr.
+ssd_status upload_table(ssd_ctx *c, cudaStream_t stream)
+{
+    const size_t T = c->offsets.size();
+    c->table_image.assign(table_bytes(c), 0);
+    int64_t *end = reinterpret_cast<int64_t *>(c->table_image.data());
+    float4 *scal = reinterpret_cast<float4 *>(c->table_image.data() + table_end_bytes(c));
+    for (size_t t = 0; t < T; ++t) {
+        end[t] = t + 1 < T ? c->offsets[t + 1] : c->n;
+        const float lr_t = c->hp.lr * c->lr_mult[t];
+        const float wd_t = c->hp.wd * c->wd_mult[t];
+        const float lr_loc_t = c->hp.lr_local * c->lr_mult[t];
+        scal[t] = make_float4(lr_t, wd_t, lr_loc_t, derive_sync_scale(lr_t, c->hp.momentum, c->hp.delay_k));
+    }
+    ssd_status st = ensure_device(c);
+    if (st != SSD_OK) return st;
+    // the image is pageable host memory: the call returns once it has been staged
+    cudaError_t e = cudaMemcpyAsync(c->tensor_table, c->table_image.data(), c->table_image.size(),
+                                    cudaMemcpyHostToDevice, stream);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    return SSD_OK;
+}
+
 ssd_status check_grads(const ssd_ctx *c, const void *const *grads)
 {
     if (!grads) return SSD_ERR_ARG;
@@ -217,15 +261,24 @@ ssd_status check_grads(const ssd_ctx *c, const void *const *grads)
     return SSD_OK;
 }
 
-template <int GT, int VW>
+template <int GT, int VW, bool PT>
 ssd_status launch_sync_b(ssd_ctx *c, const SyncParams &p, const Shape &sh, cudaStream_t stream)
 {
     switch (sh.batch) {
-    case 1: return launch(c, sync_kernel<GT, VW, 1>, p, c->n, sh, stream);
-    case 2: return launch(c, sync_kernel<GT, VW, 2>, p, c->n, sh, stream);
-    case 4: return launch(c, sync_kernel<GT, VW, 4>, p, c->n, sh, stream);
-    default: return launch(c, sync_kernel<GT, VW, 8>, p, c->n, sh, stream);
+    case 1: return launch(c, sync_kernel<GT, VW, 1, PT>, p, c->n, sh, stream);
+    case 2: return launch(c, sync_kernel<GT, VW, 2, PT>, p, c->n, sh, stream);
+    case 4: return launch(c, sync_kernel<GT, VW, 4, PT>, p, c->n, sh, stream);
+    default: return launch(c, sync_kernel<GT, VW, 8, PT>, p, c->n, sh, stream);
     }
+}
+
+template <bool PT>
+ssd_status launch_sync_t(ssd_ctx *c, const SyncParams &p, const Shape &sh, cudaStream_t stream)
+{
+    const bool bf16 = c->hp.grad_dtype == SSD_BF16;
+    if (sh.vw == 8)
+        return bf16 ? launch_sync_b<kBF16, 8, PT>(c, p, sh, stream) : launch_sync_b<kF32, 8, PT>(c, p, sh, stream);
+    return bf16 ? launch_sync_b<kBF16, 4, PT>(c, p, sh, stream) : launch_sync_b<kF32, 4, PT>(c, p, sh, stream);
 }
 
 ssd_status launch_sync(ssd_ctx *c, const void *const *grads, int flags, cudaStream_t stream)
@@ -242,11 +295,20 @@ ssd_status launch_sync(ssd_ctx *c, const void *const *grads, int flags, cudaStre
     p.flags = flags;
     p.s = c->s;
     const bool state32 = (flags & kCopy) ? c->state32 : (aligned32(c->w) && aligned32(c->mom));
+    p.tt = table_of(c);
     const Shape sh = sync_shape(c, can_use_256bit(c, state32, grads, c->hp.K));
+    return p.tt.T ? launch_sync_t<true>(c, p, sh, stream) : launch_sync_t<false>(c, p, sh, stream);
+}
+
+template <bool PT>
+ssd_status launch_glu_t(ssd_ctx *c, const GluParams &p, const Shape &sh, cudaStream_t stream)
+{
     const bool bf16 = c->hp.grad_dtype == SSD_BF16;
     if (sh.vw == 8)
-        return bf16 ? launch_sync_b<kBF16, 8>(c, p, sh, stream) : launch_sync_b<kF32, 8>(c, p, sh, stream);
-    return bf16 ? launch_sync_b<kBF16, 4>(c, p, sh, stream) : launch_sync_b<kF32, 4>(c, p, sh, stream);
+        return bf16 ? launch(c, glu_kernel<kBF16, 8, PT>, p, c->n, sh, stream)
+                    : launch(c, glu_kernel<kF32, 8, PT>, p, c->n, sh, stream);
+    return bf16 ? launch(c, glu_kernel<kBF16, 4, PT>, p, c->n, sh, stream)
+                : launch(c, glu_kernel<kF32, 4, PT>, p, c->n, sh, stream);
 }
 
 ssd_status launch_glu(ssd_ctx *c, int worker, const void *grad, int flags, cudaStream_t stream)
@@ -260,23 +322,28 @@ ssd_status launch_glu(ssd_ctx *c, int worker, const void *grad, int flags, cudaS
     p.n = c->n;
     p.flags = flags;
     p.s = c->s;
+    p.tt = table_of(c);
     const Shape sh = glu_shape(c, can_use_256bit(c, c->state32, &grad, 1));
-    const bool bf16 = c->hp.grad_dtype == SSD_BF16;
-    if (sh.vw == 8)
-        return bf16 ? launch(c, glu_kernel<kBF16, 8>, p, c->n, sh, stream)
-                    : launch(c, glu_kernel<kF32, 8>, p, c->n, sh, stream);
-    return bf16 ? launch(c, glu_kernel<kBF16, 4>, p, c->n, sh, stream)
-                : launch(c, glu_kernel<kF32, 4>, p, c->n, sh, stream);
+    return p.tt.T ? launch_glu_t<true>(c, p, sh, stream) : launch_glu_t<false>(c, p, sh, stream);
 }
 
-template <int GT, int VW>
+template <int GT, int VW, bool PT>
 ssd_status launch_step_b(ssd_ctx *c, const StepParams &p, const Shape &sh, cudaStream_t stream)
 {
     switch (sh.batch) {
-    case 1: return launch(c, step_kernel<GT, VW, 1>, p, c->n, sh, stream);
-    case 2: return launch(c, step_kernel<GT, VW, 2>, p, c->n, sh, stream);
-    default: return launch(c, step_kernel<GT, VW, 4>, p, c->n, sh, stream);
+    case 1: return launch(c, step_kernel<GT, VW, 1, PT>, p, c->n, sh, stream);
+    case 2: return launch(c, step_kernel<GT, VW, 2, PT>, p, c->n, sh, stream);
+    default: return launch(c, step_kernel<GT, VW, 4, PT>, p, c->n, sh, stream);
     }
+}
+
+template <bool PT>
+ssd_status launch_step_t(ssd_ctx *c, const StepParams &p, const Shape &sh, cudaStream_t stream)
+{
+    const bool bf16 = c->hp.grad_dtype == SSD_BF16;
+    if (sh.vw == 8)
+        return bf16 ? launch_step_b<kBF16, 8, PT>(c, p, sh, stream) : launch_step_b<kF32, 8, PT>(c, p, sh, stream);
+    return bf16 ? launch_step_b<kBF16, 4, PT>(c, p, sh, stream) : launch_step_b<kF32, 4, PT>(c, p, sh, stream);
 }
 
 ssd_status launch_step(ssd_ctx *c, const void *const *grads, int flags, cudaStream_t stream)
@@ -294,11 +361,9 @@ ssd_status launch_step(ssd_ctx *c, const void *const *grads, int flags, cudaStre
     p.K = c->hp.K;
     p.flags = flags;
     p.s = c->s;
+    p.tt = table_of(c);
     const Shape sh = step_shape(c, flags, can_use_256bit(c, c->state32, grads, c->hp.K));
-    const bool bf16 = c->hp.grad_dtype == SSD_BF16;
-    if (sh.vw == 8)
-        return bf16 ? launch_step_b<kBF16, 8>(c, p, sh, stream) : launch_step_b<kF32, 8>(c, p, sh, stream);
-    return bf16 ? launch_step_b<kBF16, 4>(c, p, sh, stream) : launch_step_b<kF32, 4>(c, p, sh, stream);
+    return p.tt.T ? launch_step_t<true>(c, p, sh, stream) : launch_step_t<false>(c, p, sh, stream);
 }
 
 ssd_status launch_copy(ssd_ctx *c, int first_worker, int count, cudaStream_t stream)
@@ -553,7 +618,46 @@ ssd_status ssd_set_counters(ssd_ctx *ctx, int64_t iter, int64_t loc_update)
     return SSD_OK;
 }
 
-ssd_status ssd_set_lr(ssd_ctx *ctx, float lr, float lr_local)
+ssd_status ssd_tensor_table_bytes(const ssd_ctx *ctx, int64_t *bytes)
+{
+    if (!ctx || !bytes) return SSD_ERR_ARG;
+    *bytes = static_cast<int64_t>(table_bytes(ctx));
+    return SSD_OK;
+}
+
+ssd_status ssd_set_tensor_scales(ssd_ctx *ctx, const float *lr_mult, const float *wd_mult,
+                                 void *device_table, void *cuda_stream)
+{
+    if (!ctx) return SSD_ERR_ARG;
+    if (!device_table) {                       // back to uniform hyper-parameters
+        ctx->tensor_table = nullptr;
+        ctx->lr_mult.clear();
+        ctx->wd_mult.clear();
+        return SSD_OK;
+    }
+    if (!aligned16(device_table)) return SSD_ERR_ALIGN;
+    const size_t T = ctx->offsets.size();
+    for (size_t t = 0; t < T; ++t) {
+        if (lr_mult && (!(lr_mult[t] > 0.0f) || !std::isfinite(lr_mult[t]))) return SSD_ERR_ARG;
+        if (wd_mult && !std::isfinite(wd_mult[t])) return SSD_ERR_ARG;
+    }
+    std::vector<float> lm(T, 1.0f), wm(T, 1.0f);
+    if (lr_mult) lm.assign(lr_mult, lr_mult + T);
+    if (wd_mult) wm.assign(wd_mult, wd_mult + T);
+    void *old_table = ctx->tensor_table;
+    ctx->lr_mult.swap(lm);
+    ctx->wd_mult.swap(wm);
+    ctx->tensor_table = device_table;
+    ssd_status st = upload_table(ctx, static_cast<cudaStream_t>(cuda_stream));
+    if (st != SSD_OK) {
+        ctx->lr_mult.swap(lm);
+        ctx->wd_mult.swap(wm);
+        ctx->tensor_table = old_table;
+    }
+    return st;
+}
+
+ssd_status ssd_set_lr(ssd_ctx *ctx, float lr, float lr_local, void *cuda_stream)
 {
     if (!ctx) return SSD_ERR_ARG;
     if (!std::isnan(lr) && (!(lr > 0.0f) || !std::isfinite(lr))) return SSD_ERR_ARG;
@@ -567,6 +671,7 @@ ssd_status ssd_set_lr(ssd_ctx *ctx, float lr, float lr_local)
         ctx->hp.lr_local = lr_local;
         ctx->s.lr_loc = lr_local;
     }
+    if (ctx->tensor_table) return upload_table(ctx, static_cast<cudaStream_t>(cuda_stream));
     return SSD_OK;
 }
 

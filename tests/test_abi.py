@@ -210,3 +210,18 @@ def test_missing_library_is_a_loud_error(monkeypatch):
     monkeypatch.setattr(B, "LIB_PATH", "/nonexistent/libssd_sgd.so")
     with pytest.raises(RuntimeError, match="no fallback"):
         B.lib()
+
+
+def test_tensor_table_size_and_validation():
+    ctx = make_ctx(numels=(10, 7, 64))
+    assert ctx.ssd_tensor_table_bytes() == 32 + 3 * 16          # 3 ends padded to 16 bytes + 3 float4
+    table = 0x30000000
+    for lr_mult, wd_mult, tbl, status in (
+            ([1.0, 0.0, 1.0], None, table, B.SSD_ERR_ARG),        # a zero lr multiplier has no grad_sync scale
+            ([1.0, -1.0, 1.0], None, table, B.SSD_ERR_ARG),
+            (None, [1.0, math.inf, 0.0], table, B.SSD_ERR_ARG),
+            (None, None, table + 8, B.SSD_ERR_ALIGN)):
+        with pytest.raises(B.SsdError) as e:
+            ctx.ssd_set_tensor_scales(lr_mult, wd_mult, tbl)
+        assert e.value.status == status
+    ctx.ssd_set_tensor_scales(None, None, None)                  # uniform: nothing to upload

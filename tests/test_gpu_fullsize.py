@@ -30,13 +30,22 @@ def sample_indices(lay, n_random=4096, seed=5):
     return np.unique(np.concatenate(picks)).astype(np.int64)
 
 
-def run_sampled(layout_name, K, W, k, iters, sigma, lr, m):
+def run_sampled(layout_name, K, W, k, iters, sigma, lr, m, per_tensor=False):
     lay = synth.get_layout(layout_name)
-    ohp, chp = make_hp(K, lr, m, W, k)
+    ohp, chp = make_hp(K, lr, m, W, k, wd=5e-4 if per_tensor else 0.0)
     idx = sample_indices(lay)
     tidx = torch.from_numpy(idx)
     w0 = synth.init_weights(lay, device="cuda")
     dev = DeviceState(lay.numels, chp, w0)
+    if per_tensor:
+        # no weight decay on BN and bias tensors, a tenth of the learning rate on the classifier
+        wd_mult = [1.0 if kind == "he" else 0.0 for kind in lay.kinds]
+        lr_mult = [0.1 if name.startswith("fc") else 1.0 for name in lay.names]
+        ends = [lay.offsets[t + 1] if t + 1 < lay.num_tensors else lay.padded_numel
+                for t in range(lay.num_tensors)]
+        ohp.set_tensor_scales(ends, lr_mult, wd_mult, arena_index=idx)
+        table = torch.empty(dev.ctx.ssd_tensor_table_bytes(), dtype=torch.uint8, device="cuda")
+        dev.ctx.ssd_set_tensor_scales(lr_mult, wd_mult, table)
     ref = oracle.State(ohp, w0[tidx.cuda()].cpu().numpy())
     mask = synth.valid_mask(lay, "cuda") if lay.padded_numel != lay.numel else None
     for n in range(iters):
@@ -75,6 +84,10 @@ def test_config_resnet50_K8_every_element():
 @pytest.mark.parametrize("k", [2, 8])
 def test_config_resnet50_K8_other_delays_sampled(k):
     run_sampled("resnet50", 8, 8, k, 50, 1e-3, 0.1, 0.9)
+
+
+def test_config_resnet50_K8_per_tensor_hyper_parameters_sampled():
+    run_sampled("resnet50", 8, 8, 4, 24, 1e-3, 0.1, 0.9, per_tensor=True)
 
 
 def test_config_vgg16_K16_sampled():

@@ -274,3 +274,67 @@ def test_every_kernel_shape_and_alignment_gives_the_same_bits(bf16):
         gpu_iteration(state, gs, "fused")
     torch.cuda.synchronize()
     compare_states(state, ref, "misaligned state")
+
+
+def tensor_ends(lay):
+    offs = lay.offsets
+    return [offs[t + 1] if t + 1 < lay.num_tensors else lay.padded_numel for t in range(lay.num_tensors)]
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+@pytest.mark.parametrize("mode", ["fused", "split"])
+def test_per_tensor_scales_and_lr_schedule(mode, bf16):
+    # tensors of odd sizes so that 8-element vectors straddle tensor boundaries; decay only on some
+    # tensors, a larger lr on others; the lr drops in the middle of the delay stage
+    K, W, k, iters = 3, 2, 3, 12
+    lay = synth.Layout("t")
+    for n in (5, 1, 10, 3, 64, 7, 1024, 2, 36, 4100):
+        lay.add("x", n, "he", 16)
+    T = lay.num_tensors
+    lr_mult = [1.0, 0.5, 2.0, 1.0, 0.25, 1.0, 1.0, 4.0, 1.0, 0.5]
+    wd_mult = [1.0, 0.0, 3.0, 0.0, 1.0, 0.0, 1.0, 0.0, 2.0, 1.0]
+    ohp, chp = make_hp(K, 0.1, 0.9, W, k, wd=0.01, bf16=bf16)
+    ohp.set_tensor_scales(tensor_ends(lay), lr_mult, wd_mult)
+    w0 = synth.init_weights(lay)
+    ref = oracle.State(ohp, w0.numpy())
+    for vw in (0, 4):
+        dev = DeviceState(lay.numels, chp, w0)
+        dev.ctx.ssd_set_kernel_shape(vw, 0)
+        table = torch.empty(dev.ctx.ssd_tensor_table_bytes(), dtype=torch.uint8, device="cuda")
+        dev.ctx.ssd_set_tensor_scales(lr_mult, wd_mult, table)
+        ohp.lr, ohp.lr_loc = np.float32(0.1), np.float32(4.0) * np.float32(0.1)
+        ref = oracle.State(ohp, w0.numpy())
+        for n in range(iters):
+            if n == 7:
+                dev.ctx.ssd_set_lr(0.05, 0.125)
+                ohp.lr, ohp.lr_loc = np.float32(0.05), np.float32(0.125)
+            grads = [synth.gradient(lay, n, i, 0.05, device="cuda") for i in range(K)]
+            if bf16:
+                grads = [synth.to_bf16(g) for g in grads]
+            gpu_iteration(dev, grads, mode)
+            ref.step([oracle_grad(g, bf16) for g in grads])
+            torch.cuda.synchronize()
+            compare_states(dev, ref, f"per-tensor vw={vw} iter {n}")
+
+
+def test_per_tensor_scales_can_be_switched_off_again():
+    lay = synth.get_layout("resnet20")
+    K = 2
+    ohp, chp = make_hp(K, 0.1, 0.9, 1, 2, wd=1e-3)
+    w0 = synth.init_weights(lay)
+    dev = DeviceState(lay.numels, chp, w0)
+    ref = oracle.State(ohp, w0.numpy())
+    wd_mult = [1.0 if kind == "he" else 0.0 for kind in lay.kinds]       # no decay on BN and bias
+    table = torch.empty(dev.ctx.ssd_tensor_table_bytes(), dtype=torch.uint8, device="cuda")
+    for n in range(8):
+        if n == 2:
+            dev.ctx.ssd_set_tensor_scales(None, wd_mult, table)
+            ohp.set_tensor_scales(tensor_ends(lay), [1.0] * lay.num_tensors, wd_mult)
+        if n == 6:
+            dev.ctx.ssd_set_tensor_scales(None, None, None)
+            ohp.tensor_end = None
+        grads = [synth.gradient(lay, n, i, 1e-2, device="cuda") for i in range(K)]
+        dev.ctx.ssd_step(grads)
+        ref.step([oracle_grad(g, False) for g in grads])
+    torch.cuda.synchronize()
+    compare_states(dev, ref, "per-tensor on/off")
