@@ -70,7 +70,8 @@ typedef enum {
     SSD_ERR_LAYOUT = 3,   /* empty or oversized layout, negative element count */
     SSD_ERR_STATE = 4,    /* call not valid in the context's current stage    */
     SSD_ERR_CUDA = 5,     /* the CUDA runtime reported an error on launch     */
-    SSD_ERR_NOMEM = 6     /* host allocation of the context failed            */
+    SSD_ERR_NOMEM = 6,    /* host allocation of the context failed            */
+    SSD_ERR_TOO_LARGE = 7 /* more tensors than the static per-tensor table holds */
 } ssd_status;
 
 typedef enum { SSD_F32 = 0, SSD_BF16 = 1 } ssd_dtype;
@@ -155,6 +156,38 @@ ssd_status ssd_schedule(const ssd_ctx *ctx, int64_t iter, int32_t *stage, int32_
  * Does not read or move the context's counters: it is the whole of synchronous
  * SGD when used alone.  One kernel launch. */
 ssd_status ssd_server_sync_update(ssd_ctx *ctx, const void *const *grads, void *cuda_stream);
+
+/* ssd_server_sync_update with per-tensor hyper-parameters for callers that cannot
+ * allocate device memory.  (The paper has no counterpart: this is a packaging of the
+ * server update above, not a step of the method.)
+ *
+ * Per-tensor scales normally need a device table that the caller allocates and
+ * hands to ssd_set_tensor_scales.  Some callers have no way to do that: a plugin
+ * that runs inside a host program whose memory pool has already claimed the whole
+ * GPU, a service with a fixed device-memory budget, or a section of code in which
+ * cudaMalloc is off limits because it synchronises the device.  For them the table
+ * lives in a fixed array inside this library's device image (24 KB on every GPU
+ * that loads the library, for as long as the process lives), and this call fills
+ * it and runs the server update in one go.  It calls no cudaMalloc, cudaFree or
+ * any other allocating routine.
+ *
+ * lr_mult, wd_mult: HOST arrays of num_tensors floats, as for
+ * ssd_set_tensor_scales (NULL = all 1; lr_mult > 0); they are read before the call
+ * returns.  grads, w and mom as for ssd_server_sync_update.  The result equals,
+ * bit for bit, ssd_set_tensor_scales followed by ssd_server_sync_update.  The
+ * context's own table (if any) is neither used nor changed.
+ *  - Layouts with more than SSD_STATIC_TABLE_MAX_TENSORS tensors are rejected with
+ *    SSD_ERR_TOO_LARGE before anything is enqueued.
+ *  - The first call on each device looks up the array's device address (with that
+ *    device current).  Make that first call before starting any stream capture.
+ *  - The array is shared by every context and every call in the process and keeps
+ *    what the last call wrote; each call overwrites the entries it uses.  Two calls
+ *    whose work can overlap on the GPU (different streams, or different contexts on
+ *    different streams) race on it: keep such calls on one stream or order them
+ *    with events. */
+#define SSD_STATIC_TABLE_MAX_TENSORS 1024
+ssd_status ssd_server_sync_update_static(ssd_ctx *ctx, const void *const *grads, const float *lr_mult,
+                                         const float *wd_mult, void *cuda_stream);
 
 /* One GLU call of worker `worker` (Algorithm 2 and the GLU rule of Section
  * 3.2.1, with the descent sign that the server rule and grad_sync imply):

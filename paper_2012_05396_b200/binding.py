@@ -18,7 +18,9 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 # SSD_SGD_LIBRARY selects another build of the same library (e.g. one compiled with other cache hints)
 LIB_PATH = os.environ.get("SSD_SGD_LIBRARY") or os.path.join(_HERE, "libssd_sgd.so")
 
-SSD_OK, SSD_ERR_ARG, SSD_ERR_ALIGN, SSD_ERR_LAYOUT, SSD_ERR_STATE, SSD_ERR_CUDA, SSD_ERR_NOMEM = range(7)
+(SSD_OK, SSD_ERR_ARG, SSD_ERR_ALIGN, SSD_ERR_LAYOUT, SSD_ERR_STATE, SSD_ERR_CUDA, SSD_ERR_NOMEM,
+ SSD_ERR_TOO_LARGE) = range(8)
+SSD_STATIC_TABLE_MAX_TENSORS = 1024
 SSD_F32, SSD_BF16 = 0, 1
 SSD_STAGE_WARMUP, SSD_STAGE_DELAY = 0, 1
 SSD_FLAG_FIRST, SSD_FLAG_REFRESH, SSD_FLAG_PULL, SSD_FLAG_COPY = 1, 2, 4, 8
@@ -27,7 +29,7 @@ SSD_MAX_WORKERS = 32
 
 EXPORTS = (
     "ssd_arena_numel", "ssd_init", "ssd_destroy", "ssd_tensor_offset", "ssd_schedule",
-    "ssd_server_sync_update", "ssd_worker_glu_update", "ssd_worker_local_step", "ssd_advance",
+    "ssd_server_sync_update", "ssd_server_sync_update_static", "ssd_worker_glu_update", "ssd_worker_local_step", "ssd_advance",
     "ssd_step", "ssd_step_host", "ssd_broadcast_weights", "ssd_worker_weights", "ssd_get_counters",
     "ssd_set_counters", "ssd_set_lr", "ssd_tensor_table_bytes", "ssd_set_tensor_scales", "ssd_get_hparams", "ssd_set_launch", "ssd_set_kernel_shape",
     "ssd_kernel_launches",
@@ -78,6 +80,7 @@ def lib():
             "ssd_tensor_offset": (i32, [vp, i32, P(i64)]),
             "ssd_schedule": (i32, [vp, i64, P(i32), P(i32)]),
             "ssd_server_sync_update": (i32, [vp, P(vp), vp]),
+            "ssd_server_sync_update_static": (i32, [vp, P(vp), P(C.c_float), P(C.c_float), vp]),
             "ssd_worker_glu_update": (i32, [vp, i32, vp, i32, vp]),
             "ssd_worker_local_step": (i32, [vp, i32, vp, vp]),
             "ssd_advance": (i32, [vp]),
@@ -191,6 +194,14 @@ class Context:
     def ssd_server_sync_update(self, grads: Sequence, stream=None):
         self._check(lib().ssd_server_sync_update(self._h, _ptr_table(grads), _stream(stream)),
                     "ssd_server_sync_update")
+
+    def ssd_server_sync_update_static(self, grads: Sequence, lr_mult=None, wd_mult=None, stream=None):
+        """Per-tensor server update whose table lives in the library's static device array: for
+        callers that must not allocate device memory.  lr_mult / wd_mult: sequences of floats or None."""
+        def arr(x):
+            return None if x is None else (C.c_float * len(x))(*[float(v) for v in x])
+        self._check(lib().ssd_server_sync_update_static(self._h, _ptr_table(grads), arr(lr_mult), arr(wd_mult),
+                                                        _stream(stream)), "ssd_server_sync_update_static")
 
     def ssd_worker_glu_update(self, worker: int, grad, flags: int, stream=None):
         self._check(lib().ssd_worker_glu_update(self._h, worker, _ptr(grad), flags, _stream(stream)),

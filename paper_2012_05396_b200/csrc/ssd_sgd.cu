@@ -6,6 +6,7 @@
 
 #include <cmath>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <string>
 #include <vector>
@@ -386,6 +387,39 @@ void advance(ssd_ctx *c)
     if (stage == SSD_STAGE_DELAY) c->loc_update += 1;
 }
 
+// ---------------------------------------------------------------------------
+// Per-tensor table in static device memory, for ssd_server_sync_update_static.
+// Layout: SSD_STATIC_TABLE_MAX_TENSORS tensor ends (int64), then as many float4
+// {lr, wd, lr_local, c}.  Every GPU that loads this library holds the 24 KB until
+// the process exits.  In host code the name below is only a handle for
+// cudaGetSymbolAddress; kernels get the device address that call returns.
+// ---------------------------------------------------------------------------
+constexpr size_t kStaticEndBytes = SSD_STATIC_TABLE_MAX_TENSORS * sizeof(int64_t);
+constexpr size_t kStaticTableBytes = kStaticEndBytes + SSD_STATIC_TABLE_MAX_TENSORS * sizeof(float4);
+static __device__ __align__(256) unsigned char g_static_tensor_table[kStaticTableBytes];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void *g_static_table_addr[kMaxDevices] = {};
+
+// Device address of the static table on the current device (looked up once per device).
+ssd_status static_table_address(ssd_ctx *c, unsigned char **out)
+{
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    if (dev < 0 || dev >= kMaxDevices) return SSD_ERR_ARG;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_table_addr[dev]) {
+        void *ptr = nullptr;
+        e = cudaGetSymbolAddress(&ptr, g_static_tensor_table);
+        if (e != cudaSuccess) return cuda_fail(c, e);
+        g_static_table_addr[dev] = ptr;
+    }
+    *out = static_cast<unsigned char *>(g_static_table_addr[dev]);
+    return SSD_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -493,6 +527,60 @@ ssd_status ssd_server_sync_update(ssd_ctx *ctx, const void *const *grads, void *
     ssd_status st = check_grads(ctx, grads);
     if (st != SSD_OK) return st;
     return launch_sync(ctx, grads, 0, static_cast<cudaStream_t>(cuda_stream));
+}
+
+ssd_status ssd_server_sync_update_static(ssd_ctx *ctx, const void *const *grads, const float *lr_mult,
+                                         const float *wd_mult, void *cuda_stream)
+{
+    if (!ctx) return SSD_ERR_ARG;
+    ssd_status st = check_grads(ctx, grads);
+    if (st != SSD_OK) return st;
+    const size_t T = ctx->offsets.size();
+    if (T > SSD_STATIC_TABLE_MAX_TENSORS) return SSD_ERR_TOO_LARGE;
+    for (size_t t = 0; t < T; ++t) {
+        if (lr_mult && (!(lr_mult[t] > 0.0f) || !std::isfinite(lr_mult[t]))) return SSD_ERR_ARG;
+        if (wd_mult && !std::isfinite(wd_mult[t])) return SSD_ERR_ARG;
+    }
+    st = ensure_device(ctx);
+    if (st != SSD_OK) return st;
+    unsigned char *table = nullptr;
+    st = static_table_address(ctx, &table);
+    if (st != SSD_OK) return st;
+
+    // Same per-tensor scalars as ssd_set_tensor_scales derives, written over the first T
+    // entries of the static table; entries beyond T keep older contents and are never read.
+    std::vector<int64_t> end(T);
+    std::vector<float4> scal(T);
+    for (size_t t = 0; t < T; ++t) {
+        end[t] = t + 1 < T ? ctx->offsets[t + 1] : ctx->n;
+        const float lm = lr_mult ? lr_mult[t] : 1.0f, wm = wd_mult ? wd_mult[t] : 1.0f;
+        const float lr_t = ctx->hp.lr * lm;
+        const float wd_t = ctx->hp.wd * wm;
+        const float lr_loc_t = ctx->hp.lr_local * lm;
+        scal[t] = make_float4(lr_t, wd_t, lr_loc_t, derive_sync_scale(lr_t, ctx->hp.momentum, ctx->hp.delay_k));
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    // pageable sources: each call returns once its bytes have been staged
+    cudaError_t e = cudaMemcpyAsync(table, end.data(), T * sizeof(int64_t), cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(table + kStaticEndBytes, scal.data(), T * sizeof(float4), cudaMemcpyHostToDevice,
+                            stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+
+    SyncParams p{};
+    for (int i = 0; i < ctx->hp.K; ++i) p.g[i] = grads[i];
+    p.w = ctx->w;
+    p.mom = ctx->mom;
+    p.n = ctx->n;
+    p.K = ctx->hp.K;
+    p.flags = 0;
+    p.s = ctx->s;
+    p.tt.end = reinterpret_cast<const int64_t *>(table);
+    p.tt.scal = reinterpret_cast<const float4 *>(table + kStaticEndBytes);
+    p.tt.T = static_cast<int>(T);
+    const bool state32 = aligned32(ctx->w) && aligned32(ctx->mom);
+    const Shape sh = sync_shape(ctx, can_use_256bit(ctx, state32, grads, ctx->hp.K));
+    return launch_sync_t<true>(ctx, p, sh, stream);
 }
 
 ssd_status ssd_worker_glu_update(ssd_ctx *ctx, int32_t worker, const void *grad, int32_t flags,
@@ -717,6 +805,7 @@ const char *ssd_status_str(ssd_status status)
     case SSD_ERR_STATE: return "call not valid in the current stage";
     case SSD_ERR_CUDA: return "CUDA runtime error";
     case SSD_ERR_NOMEM: return "out of host memory";
+    case SSD_ERR_TOO_LARGE: return "more tensors than the static table holds (SSD_STATIC_TABLE_MAX_TENSORS)";
     }
     return "unknown status";
 }
