@@ -59,13 +59,15 @@ def kernel_digest() -> str:
     return h.hexdigest()[:16]
 
 
-def step_bytes_per_param(K: int, sg: int, flags: int) -> int:
+def step_bytes_per_param(K: int, sg: int, flags: int, shared_pre: bool = False) -> int:
     """Algorithmic bytes one fused delay-stage step moves per parameter: K gradients, K local
     weights read and written, K pre_weights read, w and mom read and written; a refresh adds K
-    pre_weight stores, a pull adds K device-weight stores (and trades nothing else)."""
-    b = K * (sg + 12) + 16
+    pre_weight stores, a pull adds K device-weight stores (and trades nothing else).  With one
+    shared pre_weight buffer it is read once and refreshed once instead of K times."""
+    pre_copies = 1 if shared_pre else K
+    b = K * (sg + 8) + 4 * pre_copies + 16
     if flags & 2:       # refresh
-        b += 4 * K
+        b += 4 * pre_copies
     if flags & 4:       # pull
         b += 4 * K
     return b
@@ -225,6 +227,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--per-tensor", action="store_true",
                     help="per-tensor hyper-parameters: weight decay 5e-4 on conv/FC weights only")
+    ap.add_argument("--shared-pre", action="store_true",
+                    help="one pre_weight buffer shared by all workers (fewer algorithmic bytes, counted as such)")
     ap.add_argument("--threads", type=int, default=0, help="threads per block (0 = library default)")
     ap.add_argument("--blocks-per-sm", type=int, default=0, help="resident blocks per SM (0 = default)")
     args = ap.parse_args()
@@ -265,7 +269,7 @@ def main():
     hp = B.make_hparams(K, wl["lr"], wl["m"], wl["W"], wl["k"], wd=5e-4 if args.per_tensor else 0.0,
                         lr_local=nan, alpha=nan, beta=nan, rescale=nan, grad_dtype=B.SSD_F32)
     w0 = synth.init_weights(lay, device=dev_name)
-    st = DeviceState(lay.numels, hp, w0, device=dev_name, fill=0.0)
+    st = DeviceState(lay.numels, hp, w0, device=dev_name, fill=0.0, shared_pre=args.shared_pre)
     if args.per_tensor:
         table = torch.empty(st.ctx.ssd_tensor_table_bytes(), dtype=torch.uint8, device=dev_name)
         st.ctx.ssd_set_tensor_scales(None, [1.0 if kind == "he" else 0.0 for kind in lay.kinds], table)
@@ -309,12 +313,12 @@ def main():
     total_ms = ev[0].elapsed_time(ev[-1])
     per_launch_ms = [ev[n].elapsed_time(ev[n + 1]) for n in range(args.steps)]
     total_ms = max_over_ranks(total_ms, dev_name, world)
-    bytes_per_launch = [step_bytes_per_param(K, sg, f) * N for f in flags_of]
+    bytes_per_launch = [step_bytes_per_param(K, sg, f, args.shared_pre) * N for f in flags_of]
     value = whole_job_rate(float(sum(bytes_per_launch)), world, total_ms) / 1e9
     peak, peak_kind = measured_peak()
     achieved = (sum(bytes_per_launch) / len(bytes_per_launch)) / (statistics.mean(per_launch_ms) * 1e-3) / 1e9
     traffic = None
-    if NCU_TRAFFIC["digest"] == kernel_digest() and NCU_TRAFFIC["K"] == K and sg == 4:
+    if NCU_TRAFFIC["digest"] == kernel_digest() and NCU_TRAFFIC["K"] == K and sg == 4 and not args.shared_pre:
         per = NCU_TRAFFIC["bytes_per_param"]
         if all((f & 6) in per for f in flags_of):
             traffic = N * statistics.mean(per[f & 6] for f in flags_of)
@@ -330,6 +334,7 @@ def main():
                    "workers": K, "delay_k": wl["k"], "ssd_warmup_iters": wl["W"], "grad_dtype": "f32",
                    "stage": "steps-delay", "kernel": "fused ssd_step", "replicas": world,
                    "hyper_parameters": "per tensor" if args.per_tensor else "uniform",
+                   "pre_weight": "one shared buffer" if args.shared_pre else "one buffer per worker",
                    "device_bytes": st.bytes() + n_sets * K * N * sg,
                    "l2": "inputs larger than L2 (no flush needed)"
                    if st.bytes() > 4 * 126e6 else "L2-resident: not an HBM measurement"},
@@ -364,7 +369,7 @@ def main():
         torch.cuda.synchronize()
         e_ms = e0.elapsed_time(e1)
         e_ms = max_over_ranks(e_ms, dev_name, world)
-        e_bytes = float(sum(step_bytes_per_param(K, sg, f) * N for f in e_flags))
+        e_bytes = float(sum(step_bytes_per_param(K, sg, f, args.shared_pre) * N for f in e_flags))
         e2e = {"value": whole_job_rate(e_bytes, world, e_ms) / 1e9, "unit": UNIT, "h2d_bytes_per_step": K * N * sg,
                "d2h_bytes_per_step": N * 4, "steps": args.e2e_steps, "ms_per_step": e_ms / args.e2e_steps,
                "call": "ssd_step_host"}

@@ -106,7 +106,14 @@ typedef struct {
 /* Caller-owned device state.  w_loc, pre, w_dev: host arrays of K device pointers.
  * The K*3+2 buffers must not overlap each other or any gradient buffer.  With
  * delay_k == 0 (synchronous SGD only) no worker state is ever touched and the
- * three tables may be NULL. */
+ * three tables may be NULL.
+ * Shared pre_weight: the K pre_weight buffers always hold equal values (each worker
+ * sets its own from the same pulled global weight: "the same pre_weight", Section
+ * 3.3), so all K entries of `pre` may point at ONE buffer.  ssd_step then reads it
+ * once per element instead of K times and writes it once (K-1 arenas less memory,
+ * 4(K-1) bytes per parameter less traffic); results are unchanged.  The per-worker
+ * calls (ssd_worker_glu_update, ssd_worker_local_step in the delay stage) would
+ * overwrite it between workers and return SSD_ERR_STATE for such a context. */
 typedef struct {
     float *w;                     /* global weight w_t (server)                 */
     float *mom;                   /* server momentum mom_t                      */

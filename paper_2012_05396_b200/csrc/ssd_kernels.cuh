@@ -82,6 +82,7 @@ struct StepParams {
     float *w, *mom;
     int64_t n;
     int K, flags;
+    int shared_pre;                // 1: pre[0] is the one pre_weight of all workers
     Scalars s;
     TensorTable tt;
 };
@@ -313,6 +314,12 @@ __device__ __forceinline__ void step_at(const StepParams &p, int64_t e)
     Vec<VW> w = ld_f32<VW>(p.w, e);
     Vec<VW> mom = ld_f32<VW>(p.mom, e);
     Vec<VW> sum;
+    // A shared pre_weight is read once per element instead of once per worker, and written
+    // once: on the iterations that write it every worker's local weight holds the same pulled
+    // global weight, so worker 0's value is everyone's.
+    const bool shared = p.shared_pre != 0;
+    Vec<VW> pre_shared;
+    if (shared && !first) pre_shared = ld_f32<VW>(p.pre[0], e);
     GroupScalars<PT, VW> sc(p.s, p.tt, e);
     for (int i0 = 0; i0 < p.K; i0 += B) {
         Grad<GT, VW> g[B];
@@ -322,7 +329,7 @@ __device__ __forceinline__ void step_at(const StepParams &p, int64_t e)
             if (i0 + b < p.K) {
                 g[b] = ld_grad<GT, VW>(p.g[i0 + b], e);
                 wl[b] = ld_f32<VW>(p.w_loc[i0 + b], e);
-                if (!first) pr[b] = ld_f32<VW>(p.pre[i0 + b], e);
+                if (!first && !shared) pr[b] = ld_f32<VW>(p.pre[i0 + b], e);
             }
         }
 #pragma unroll
@@ -334,9 +341,10 @@ __device__ __forceinline__ void step_at(const StepParams &p, int64_t e)
                 for (int l = 0; l < VW; ++l) {
                     const float gl = g[b].get(l);
                     sum.v[l] = (i == 0) ? gl : __fadd_rn(sum.v[l], gl);
-                    r.v[l] = glu_elem(gl, wl[b].v[l], first ? wl[b].v[l] : pr[b].v[l], sc.at(l));
+                    const float pl = first ? wl[b].v[l] : shared ? pre_shared.v[l] : pr[b].v[l];
+                    r.v[l] = glu_elem(gl, wl[b].v[l], pl, sc.at(l));
                 }
-                if (first || refresh) st_f32<VW>(p.pre[i], e, wl[b]);
+                if ((first || refresh) && (!shared || i == 0)) st_f32<VW>(p.pre[i], e, wl[b]);
                 st_f32<VW>(pull ? p.w_dev[i] : p.w_loc[i], e, r);
             }
         }

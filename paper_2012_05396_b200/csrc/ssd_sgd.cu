@@ -33,6 +33,7 @@ struct ssd_ctx {
     float *w = nullptr, *mom = nullptr;
     float *w_loc[kMaxWorkers]{}, *pre[kMaxWorkers]{}, *w_dev[kMaxWorkers]{};
     bool has_workers = true;          // false: delay_k == 0 and no worker tables were given
+    bool shared_pre = false;          // all K pre_weight pointers are the same buffer
     int64_t iter = 0, loc_update = 0;
     bool state32 = false;             // every state buffer is 32-byte aligned
     int threads = 0, blocks_per_sm = 0;     // 0: the kernel's default shape
@@ -361,6 +362,7 @@ ssd_status launch_step(ssd_ctx *c, const void *const *grads, int flags, cudaStre
     p.n = c->n;
     p.K = c->hp.K;
     p.flags = flags;
+    p.shared_pre = c->shared_pre ? 1 : 0;
     p.s = c->s;
     p.tt = table_of(c);
     const Shape sh = step_shape(c, flags, can_use_256bit(c, c->state32, grads, c->hp.K));
@@ -457,10 +459,14 @@ ssd_status ssd_init(ssd_ctx **out, const ssd_layout *layout, const ssd_hparams *
         delete c;
         return st;
     }
+    // All K pre_weight pointers equal: one shared pre_weight (its K copies always hold the same
+    // values, every worker takes it from the same pulled global weight).
+    bool shared_pre = workers && hp->K > 1 && b->pre[0] != nullptr;
+    for (int i = 1; shared_pre && i < hp->K; ++i) shared_pre = b->pre[i] == b->pre[0];
     std::vector<const void *> all{b->w, b->mom};
     for (int i = 0; workers && i < hp->K; ++i) {
         all.push_back(b->w_loc[i]);
-        all.push_back(b->pre[i]);
+        if (!shared_pre || i == 0) all.push_back(b->pre[i]);
         all.push_back(b->w_dev[i]);
     }
     for (const void *p : all) {
@@ -493,6 +499,7 @@ ssd_status ssd_init(ssd_ctx **out, const ssd_layout *layout, const ssd_hparams *
     c->w = b->w;
     c->mom = b->mom;
     c->has_workers = workers;
+    c->shared_pre = shared_pre;
     c->state32 = true;
     for (const void *p : all) c->state32 = c->state32 && aligned32(p);
     for (int i = 0; workers && i < hp->K; ++i) {
@@ -590,6 +597,7 @@ ssd_status ssd_worker_glu_update(ssd_ctx *ctx, int32_t worker, const void *grad,
     if (worker < 0 || worker >= ctx->hp.K) return SSD_ERR_ARG;
     if (flags & ~(SSD_FLAG_FIRST | SSD_FLAG_REFRESH | SSD_FLAG_PULL)) return SSD_ERR_ARG;
     if (ctx->hp.delay_k == 0) return SSD_ERR_STATE;
+    if (ctx->shared_pre) return SSD_ERR_STATE;
     if (!aligned16(grad)) return SSD_ERR_ALIGN;
     return launch_glu(ctx, worker, grad, flags, static_cast<cudaStream_t>(cuda_stream));
 }
@@ -606,6 +614,7 @@ ssd_status ssd_worker_local_step(ssd_ctx *ctx, int32_t worker, const void *grad,
         return SSD_OK;
     }
     if (!grad) return SSD_ERR_ARG;
+    if (ctx->shared_pre) return SSD_ERR_STATE;
     if (!aligned16(grad)) return SSD_ERR_ALIGN;
     return launch_glu(ctx, worker, grad, flags, stream);
 }

@@ -16,7 +16,8 @@ class DeviceState:
     """
 
     def __init__(self, numels: Sequence[int], hp: B.ssd_hparams, w0: torch.Tensor,
-                 device="cuda", fill: float = float("nan"), worker_state: bool = True):
+                 device="cuda", fill: float = float("nan"), worker_state: bool = True,
+                 shared_pre: bool = False):
         self.numels = [int(n) for n in numels]
         self.n = B.ssd_arena_numel(self.numels)
         assert w0.numel() == self.n and w0.dtype == torch.float32
@@ -32,8 +33,9 @@ class DeviceState:
             return
         # Algorithm 1 starts with every worker pulling w_0.
         self.w_loc = [self.w.clone() for _ in range(self.K)]
+        # shared_pre: one pre_weight buffer for all workers (K references to the same tensor)
         self.pre = [torch.full((self.n,), fill, dtype=torch.float32, device=self.device)
-                    for _ in range(self.K)]
+                    for _ in range(1 if shared_pre else self.K)] * (self.K if shared_pre else 1)
         self.w_dev = [torch.full((self.n,), fill, dtype=torch.float32, device=self.device)
                       for _ in range(self.K)]
         self.ctx = B.Context(self.numels, hp, self.w, self.mom, self.w_loc, self.pre, self.w_dev)
@@ -44,4 +46,4 @@ class DeviceState:
         return (self.w, self.w_loc[i], self.w_dev[i])[view]
 
     def bytes(self) -> int:
-        return (2 + len(self.w_loc) + len(self.pre) + len(self.w_dev)) * self.n * 4
+        return (2 + len(self.w_loc) + len({t.data_ptr() for t in self.pre}) + len(self.w_dev)) * self.n * 4

@@ -102,7 +102,16 @@ def test_init_rejects_bad_pointers():
         B.Context([16], hp, w, mom, wl, [pre[0], None], wdv)
     assert e.value.status == B.SSD_ERR_ARG
     with pytest.raises(B.SsdError) as e:                  # two state buffers at one address
-        B.Context([16], hp, w, mom, wl, [pre[0], pre[0]], wdv)
+        B.Context([16], hp, w, mom, [wl[0], wl[0]], pre, wdv)
+    assert e.value.status == B.SSD_ERR_ARG
+    with pytest.raises(B.SsdError) as e:
+        B.Context([16], hp, w, mom, wl, [pre[0], wl[1]], wdv)
+    assert e.value.status == B.SSD_ERR_ARG
+    B.Context([16], hp, w, mom, wl, [pre[0], pre[0]], wdv)   # one shared pre_weight for all workers: allowed
+    hp3 = B.make_hparams(3, 0.1, 0.9, 2, 4)
+    w3, mom3, wl3, pre3, wdv3 = fake_ptrs(3)
+    with pytest.raises(B.SsdError) as e:                  # shared by some workers only
+        B.Context([16], hp3, w3, mom3, wl3, [pre3[0], pre3[0], pre3[2]], wdv3)
     assert e.value.status == B.SSD_ERR_ARG
     L = B.lib()
     assert L.ssd_init(None, None, None, None) == B.SSD_ERR_ARG

@@ -338,3 +338,33 @@ def test_per_tensor_scales_can_be_switched_off_again():
         ref.step([oracle_grad(g, False) for g in grads])
     torch.cuda.synchronize()
     compare_states(dev, ref, "per-tensor on/off")
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_shared_pre_weight_gives_the_same_results(bf16):
+    # one pre_weight buffer for all K workers: ssd_step reads it once per element; every worker's
+    # pre_weight in the oracle must equal it
+    K, W, k, iters = 5, 2, 3, 13
+    lay = synth.get_layout("resnet20")
+    ohp, chp = make_hp(K, 0.1, 0.9, W, k, wd=1e-3, bf16=bf16)
+    w0 = synth.init_weights(lay)
+    for vw, batch in ((0, 0), (4, 4), (8, 2)):
+        dev = DeviceState(lay.numels, chp, w0, shared_pre=True)
+        assert len({t.data_ptr() for t in dev.pre}) == 1
+        dev.ctx.ssd_set_kernel_shape(vw, batch)
+        ref = oracle.State(ohp, w0.numpy())
+        for n in range(iters):
+            grads = [synth.gradient(lay, n, i, 1e-2, device="cuda") for i in range(K)]
+            if bf16:
+                grads = [synth.to_bf16(g) for g in grads]
+            dev.ctx.ssd_step(grads)
+            ref.step([oracle_grad(g, bf16) for g in grads])
+            torch.cuda.synchronize()
+            compare_states(dev, ref, f"shared pre vw={vw} iter {n}")
+    # the per-worker calls cannot be used with a shared pre_weight
+    with pytest.raises(B.SsdError) as e:
+        dev.ctx.ssd_worker_glu_update(0, grads[0], 0)
+    assert e.value.status == B.SSD_ERR_STATE
+    with pytest.raises(B.SsdError) as e:
+        dev.ctx.ssd_worker_local_step(0, grads[0])
+    assert e.value.status == B.SSD_ERR_STATE
