@@ -200,14 +200,10 @@ Shape sync_shape(const ssd_ctx *c, bool wide_ok)
 
 Shape step_shape(const ssd_ctx *c, int flags, bool wide_ok)
 {
-    const int K = c->hp.K;
-    Shape sh;
-    if (flags & (kRefresh | kPull | kFirst))
-        sh = Shape{8, 1, 128, 4};          // write-heavy iterations: 512 threads per SM
-    else if (c->hp.grad_dtype == SSD_BF16)
-        sh = Shape{8, 1, 128, 5};
-    else
-        sh = Shape{8, 1, 128, K >= 16 ? 6 : 5};
+    // Iterations that add K stores per element (pull; refresh or first call with one pre_weight
+    // per worker) are write-heavy: 512 threads per SM.  The others: 640 threads per SM.
+    const bool k_extra_stores = (flags & kPull) || (!c->shared_pre && (flags & (kRefresh | kFirst)));
+    const Shape sh = k_extra_stores ? Shape{8, 1, 128, 4} : Shape{8, 1, 128, 5};
     return finish_shape(c, sh, wide_ok, 4);
 }
 
