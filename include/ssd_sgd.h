@@ -233,12 +233,16 @@ ssd_status ssd_advance(ssd_ctx *ctx);
 ssd_status ssd_step(ssd_ctx *ctx, const void *const *grads, void *cuda_stream);
 
 /* ssd_step for gradients that arrive in HOST memory (as they would from a
- * network push).  `host_grads`: K host pointers (pinned memory for asynchronous
- * copies); `staging`: K device buffers of arena size (gradient dtype) that
+ * network push).  `host_grads`: K host pointers (pinned memory, or the copies are
+ * not asynchronous); `staging`: K device buffers of arena size (gradient dtype) that
  * receive them; `host_w_out`: optional host buffer that receives the new global
- * weight w (NULL = no read-back).  Enqueues K host-to-device copies, the step and
- * the device-to-host copy on `cuda_stream`; the caller synchronises the stream
- * before reading host_w_out or reusing host_grads. */
+ * weight w (NULL = no read-back).  The arena is processed in chunks of 2^24
+ * elements: the host-to-device copies of one chunk, the update of the previous one
+ * and the device-to-host copy of the one before overlap, on two side streams that
+ * the context creates at the first call (driver objects, no device memory).  All of
+ * it is ordered after the work already on `cuda_stream`, and `cuda_stream` ends
+ * behind the last copy: the caller synchronises `cuda_stream` before reading
+ * host_w_out or reusing host_grads.  One kernel launch per chunk. */
 ssd_status ssd_step_host(ssd_ctx *ctx, const void *const *host_grads, void *const *staging,
                          float *host_w_out, void *cuda_stream);
 

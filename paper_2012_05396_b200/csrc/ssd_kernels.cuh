@@ -51,6 +51,7 @@ struct Scalars {
 struct TensorTable {
     const int64_t *end;
     const float4 *scal;
+    int64_t base;                  // arena position of the launch's element 0 (range launches)
     int T;
 };
 
@@ -242,10 +243,11 @@ template <bool PT, int VW> struct GroupScalars {
 #pragma unroll
         for (int q = 0; q < VW / 4; ++q) g[q] = uniform;
         if (PT) {
-            const int t = tensor_of(tt, e);
+            const int64_t pos = e + tt.base;
+            const int t = tensor_of(tt, pos);
             g[0] = with_tensor(uniform, tt, t);
             if (VW == 8)
-                g[VW / 4 - 1] = (e + 4 < __ldg(tt.end + t)) ? g[0] : with_tensor(uniform, tt, tensor_of(tt, e + 4));
+                g[VW / 4 - 1] = (pos + 4 < __ldg(tt.end + t)) ? g[0] : with_tensor(uniform, tt, tensor_of(tt, pos + 4));
         }
     }
     __device__ __forceinline__ const Scalars &at(int l) const { return g[l >> 2]; }

@@ -16,6 +16,7 @@ namespace {
 using namespace ssd;
 
 constexpr int64_t kMaxArena = int64_t(1) << 40;
+constexpr int64_t kHostChunkElems = int64_t(1) << 24;   // ssd_step_host: elements per pipelined chunk
 
 struct Device {
     bool ready = false;
@@ -42,6 +43,9 @@ struct ssd_ctx {
     std::vector<float> lr_mult, wd_mult;
     void *tensor_table = nullptr;
     std::vector<unsigned char> table_image;   // what was last uploaded
+    // ssd_step_host pipelines chunks over two side streams (copies in, copies out)
+    cudaStream_t in_stream = nullptr, out_stream = nullptr;
+    std::vector<cudaEvent_t> events;
     int64_t launches = 0;
     Device dev;
     std::string cuda_error;
@@ -192,7 +196,7 @@ Shape sync_shape(const ssd_ctx *c, bool wide_ok)
     const int K = c->hp.K;
     Shape sh;
     if (c->hp.grad_dtype == SSD_BF16)
-        sh = K >= 4 ? Shape{8, 4, 128, 6} : Shape{8, 1, 128, 4};
+        sh = K >= 4 ? Shape{8, 4, 128, 6} : Shape{8, 1, 128, K == 1 ? 4 : 6};
     else
         sh = K >= 4 ? Shape{8, 4, 128, 5} : Shape{8, 1, 128, 6};
     return finish_shape(c, sh, wide_ok, 8);
@@ -263,10 +267,10 @@ template <int GT, int VW, bool PT>
 ssd_status launch_sync_b(ssd_ctx *c, const SyncParams &p, const Shape &sh, cudaStream_t stream)
 {
     switch (sh.batch) {
-    case 1: return launch(c, sync_kernel<GT, VW, 1, PT>, p, c->n, sh, stream);
-    case 2: return launch(c, sync_kernel<GT, VW, 2, PT>, p, c->n, sh, stream);
-    case 4: return launch(c, sync_kernel<GT, VW, 4, PT>, p, c->n, sh, stream);
-    default: return launch(c, sync_kernel<GT, VW, 8, PT>, p, c->n, sh, stream);
+    case 1: return launch(c, sync_kernel<GT, VW, 1, PT>, p, p.n, sh, stream);
+    case 2: return launch(c, sync_kernel<GT, VW, 2, PT>, p, p.n, sh, stream);
+    case 4: return launch(c, sync_kernel<GT, VW, 4, PT>, p, p.n, sh, stream);
+    default: return launch(c, sync_kernel<GT, VW, 8, PT>, p, p.n, sh, stream);
     }
 }
 
@@ -279,21 +283,31 @@ ssd_status launch_sync_t(ssd_ctx *c, const SyncParams &p, const Shape &sh, cudaS
     return bf16 ? launch_sync_b<kBF16, 4, PT>(c, p, sh, stream) : launch_sync_b<kF32, 4, PT>(c, p, sh, stream);
 }
 
-ssd_status launch_sync(ssd_ctx *c, const void *const *grads, int flags, cudaStream_t stream)
+// Gradient pointer advanced by `lo` elements of the context's gradient type.
+const void *grad_at(const ssd_ctx *c, const void *g, int64_t lo)
+{
+    return static_cast<const unsigned char *>(g) + lo * (c->hp.grad_dtype == SSD_BF16 ? 2 : 4);
+}
+
+// The launch functions take an element range [lo, lo + count) of the arena (lo a multiple of 8,
+// which keeps every alignment property of the buffers); count < 0 means the whole arena.
+ssd_status launch_sync(ssd_ctx *c, const void *const *grads, int flags, cudaStream_t stream,
+                       int64_t lo = 0, int64_t count = -1)
 {
     SyncParams p{};
     for (int i = 0; i < c->hp.K; ++i) {
-        p.g[i] = grads[i];
-        p.w_loc[i] = c->w_loc[i];
+        p.g[i] = grad_at(c, grads[i], lo);
+        p.w_loc[i] = c->w_loc[i] ? c->w_loc[i] + lo : nullptr;
     }
-    p.w = c->w;
-    p.mom = c->mom;
-    p.n = c->n;
+    p.w = c->w + lo;
+    p.mom = c->mom + lo;
+    p.n = count < 0 ? c->n : count;
     p.K = c->hp.K;
     p.flags = flags;
     p.s = c->s;
     const bool state32 = (flags & kCopy) ? c->state32 : (aligned32(c->w) && aligned32(c->mom));
     p.tt = table_of(c);
+    p.tt.base = lo;
     const Shape sh = sync_shape(c, can_use_256bit(c, state32, grads, c->hp.K));
     return p.tt.T ? launch_sync_t<true>(c, p, sh, stream) : launch_sync_t<false>(c, p, sh, stream);
 }
@@ -303,10 +317,10 @@ ssd_status launch_glu_t(ssd_ctx *c, const GluParams &p, const Shape &sh, cudaStr
 {
     const bool bf16 = c->hp.grad_dtype == SSD_BF16;
     if (sh.vw == 8)
-        return bf16 ? launch(c, glu_kernel<kBF16, 8, PT>, p, c->n, sh, stream)
-                    : launch(c, glu_kernel<kF32, 8, PT>, p, c->n, sh, stream);
-    return bf16 ? launch(c, glu_kernel<kBF16, 4, PT>, p, c->n, sh, stream)
-                : launch(c, glu_kernel<kF32, 4, PT>, p, c->n, sh, stream);
+        return bf16 ? launch(c, glu_kernel<kBF16, 8, PT>, p, p.n, sh, stream)
+                    : launch(c, glu_kernel<kF32, 8, PT>, p, p.n, sh, stream);
+    return bf16 ? launch(c, glu_kernel<kBF16, 4, PT>, p, p.n, sh, stream)
+                : launch(c, glu_kernel<kF32, 4, PT>, p, p.n, sh, stream);
 }
 
 ssd_status launch_glu(ssd_ctx *c, int worker, const void *grad, int flags, cudaStream_t stream)
@@ -329,9 +343,9 @@ template <int GT, int VW, bool PT>
 ssd_status launch_step_b(ssd_ctx *c, const StepParams &p, const Shape &sh, cudaStream_t stream)
 {
     switch (sh.batch) {
-    case 1: return launch(c, step_kernel<GT, VW, 1, PT>, p, c->n, sh, stream);
-    case 2: return launch(c, step_kernel<GT, VW, 2, PT>, p, c->n, sh, stream);
-    default: return launch(c, step_kernel<GT, VW, 4, PT>, p, c->n, sh, stream);
+    case 1: return launch(c, step_kernel<GT, VW, 1, PT>, p, p.n, sh, stream);
+    case 2: return launch(c, step_kernel<GT, VW, 2, PT>, p, p.n, sh, stream);
+    default: return launch(c, step_kernel<GT, VW, 4, PT>, p, p.n, sh, stream);
     }
 }
 
@@ -344,23 +358,25 @@ ssd_status launch_step_t(ssd_ctx *c, const StepParams &p, const Shape &sh, cudaS
     return bf16 ? launch_step_b<kBF16, 4, PT>(c, p, sh, stream) : launch_step_b<kF32, 4, PT>(c, p, sh, stream);
 }
 
-ssd_status launch_step(ssd_ctx *c, const void *const *grads, int flags, cudaStream_t stream)
+ssd_status launch_step(ssd_ctx *c, const void *const *grads, int flags, cudaStream_t stream,
+                       int64_t lo = 0, int64_t count = -1)
 {
     StepParams p{};
     for (int i = 0; i < c->hp.K; ++i) {
-        p.g[i] = grads[i];
-        p.w_loc[i] = c->w_loc[i];
-        p.pre[i] = c->pre[i];
-        p.w_dev[i] = c->w_dev[i];
+        p.g[i] = grad_at(c, grads[i], lo);
+        p.w_loc[i] = c->w_loc[i] + lo;
+        p.pre[i] = c->pre[i] + lo;
+        p.w_dev[i] = c->w_dev[i] + lo;
     }
-    p.w = c->w;
-    p.mom = c->mom;
-    p.n = c->n;
+    p.w = c->w + lo;
+    p.mom = c->mom + lo;
+    p.n = count < 0 ? c->n : count;
     p.K = c->hp.K;
     p.flags = flags;
     p.shared_pre = c->shared_pre ? 1 : 0;
     p.s = c->s;
     p.tt = table_of(c);
+    p.tt.base = lo;
     const Shape sh = step_shape(c, flags, can_use_256bit(c, c->state32, grads, c->hp.K));
     return p.tt.T ? launch_step_t<true>(c, p, sh, stream) : launch_step_t<false>(c, p, sh, stream);
 }
@@ -373,8 +389,8 @@ ssd_status launch_copy(ssd_ctx *c, int first_worker, int count, cudaStream_t str
     p.n = c->n;
     p.K = count;
     const Shape sh = finish_shape(c, Shape{8, 1, 256, 0}, c->state32, 1);
-    if (sh.vw == 8) return launch(c, copy_kernel<8>, p, c->n, sh, stream);
-    return launch(c, copy_kernel<4>, p, c->n, sh, stream);
+    if (sh.vw == 8) return launch(c, copy_kernel<8>, p, p.n, sh, stream);
+    return launch(c, copy_kernel<4>, p, p.n, sh, stream);
 }
 
 void advance(ssd_ctx *c)
@@ -507,7 +523,14 @@ ssd_status ssd_init(ssd_ctx **out, const ssd_layout *layout, const ssd_hparams *
     return SSD_OK;
 }
 
-void ssd_destroy(ssd_ctx *ctx) { delete ctx; }
+void ssd_destroy(ssd_ctx *ctx)
+{
+    if (!ctx) return;
+    for (cudaEvent_t e : ctx->events) cudaEventDestroy(e);
+    if (ctx->in_stream) cudaStreamDestroy(ctx->in_stream);
+    if (ctx->out_stream) cudaStreamDestroy(ctx->out_stream);
+    delete ctx;
+}
 
 ssd_status ssd_tensor_offset(const ssd_ctx *ctx, int32_t tensor, int64_t *elem_offset)
 {
@@ -648,18 +671,61 @@ ssd_status ssd_step_host(ssd_ctx *ctx, const void *const *host_grads, void *cons
     ssd_status st = ensure_device(ctx);
     if (st != SSD_OK) return st;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const size_t gbytes = static_cast<size_t>(ctx->n) * (ctx->hp.grad_dtype == SSD_BF16 ? 2 : 4);
-    for (int i = 0; i < ctx->hp.K; ++i) {
-        cudaError_t e = cudaMemcpyAsync(staging[i], host_grads[i], gbytes, cudaMemcpyHostToDevice, stream);
-        if (e != cudaSuccess) return cuda_fail(ctx, e);
+    const int K = ctx->hp.K;
+    const size_t sg = ctx->hp.grad_dtype == SSD_BF16 ? 2 : 4;
+    int32_t stage, flags;
+    schedule_of(ctx, ctx->iter, &stage, &flags);
+
+    // The arena is cut into chunks; chunk c's gradients are copied in on a side stream while
+    // chunk c-1 is being updated on the caller's stream and chunk c-2's new weights are copied
+    // out on a second side stream.  The update is elementwise, so chunks are independent.
+    const int64_t chunk = kHostChunkElems;
+    const int chunks = static_cast<int>((ctx->n + chunk - 1) / chunk);
+    cudaError_t e = cudaSuccess;
+    if (!ctx->in_stream) e = cudaStreamCreateWithFlags(&ctx->in_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess && !ctx->out_stream) e = cudaStreamCreateWithFlags(&ctx->out_stream, cudaStreamNonBlocking);
+    while (e == cudaSuccess && ctx->events.size() < static_cast<size_t>(2 * chunks + 2)) {
+        cudaEvent_t ev;
+        e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
+        if (e == cudaSuccess) ctx->events.push_back(ev);
     }
-    st = ssd_step(ctx, const_cast<const void *const *>(staging), cuda_stream);
-    if (st != SSD_OK) return st;
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    cudaEvent_t ev_start = ctx->events[2 * chunks], ev_end = ctx->events[2 * chunks + 1];
+    // everything already enqueued on the caller's stream comes first
+    e = cudaEventRecord(ev_start, stream);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->in_stream, ev_start, 0);
+    if (e == cudaSuccess && host_w_out) e = cudaStreamWaitEvent(ctx->out_stream, ev_start, 0);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    for (int c = 0; c < chunks; ++c) {
+        const int64_t lo = static_cast<int64_t>(c) * chunk;
+        const int64_t count = ctx->n - lo < chunk ? ctx->n - lo : chunk;
+        for (int i = 0; i < K && e == cudaSuccess; ++i)
+            e = cudaMemcpyAsync(static_cast<unsigned char *>(staging[i]) + lo * sg,
+                                static_cast<const unsigned char *>(host_grads[i]) + lo * sg, count * sg,
+                                cudaMemcpyHostToDevice, ctx->in_stream);
+        if (e == cudaSuccess) e = cudaEventRecord(ctx->events[2 * c], ctx->in_stream);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, ctx->events[2 * c], 0);
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
+        st = (stage == SSD_STAGE_WARMUP)
+                 ? launch_sync(ctx, const_cast<const void *const *>(staging), flags & SSD_FLAG_COPY, stream, lo, count)
+                 : launch_step(ctx, const_cast<const void *const *>(staging), flags, stream, lo, count);
+        if (st != SSD_OK) return st;
+        if (host_w_out) {
+            e = cudaEventRecord(ctx->events[2 * c + 1], stream);
+            if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->out_stream, ctx->events[2 * c + 1], 0);
+            if (e == cudaSuccess)
+                e = cudaMemcpyAsync(host_w_out + lo, ctx->w + lo, count * sizeof(float), cudaMemcpyDeviceToHost,
+                                    ctx->out_stream);
+            if (e != cudaSuccess) return cuda_fail(ctx, e);
+        }
+    }
     if (host_w_out) {
-        cudaError_t e = cudaMemcpyAsync(host_w_out, ctx->w, static_cast<size_t>(ctx->n) * 4,
-                                        cudaMemcpyDeviceToHost, stream);
+        // the caller's stream ends behind the last copy out
+        e = cudaEventRecord(ev_end, ctx->out_stream);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, ev_end, 0);
         if (e != cudaSuccess) return cuda_fail(ctx, e);
     }
+    advance(ctx);
     return SSD_OK;
 }
 

@@ -170,3 +170,36 @@ def test_sweep_largest_size_sampled(K, bf16):
     if torch.cuda.mem_get_info()[0] < need:
         pytest.skip(f"needs {need / 2**30:.0f} GiB of free device memory")
     sweep_point(n, K, bf16, 0, sampled=True)
+
+
+def test_step_host_in_chunks_equals_one_step():
+    # An arena longer than one 2^24-element chunk: ssd_step_host pipelines two chunks over its side
+    # streams and must leave exactly the state of ssd_step on device-resident gradients (which the
+    # tests above tie to the oracle), also with per-tensor scalars, whose lookup depends on position.
+    lay = synth.get_layout("resnet50")
+    K, W, k = 2, 1, 2
+    _, chp = make_hp(K, 0.1, 0.9, W, k, wd=5e-4)
+    w0 = synth.init_weights(lay, device="cuda")
+    a, b = DeviceState(lay.numels, chp, w0), DeviceState(lay.numels, chp, w0)
+    wd_mult = [1.0 if kind == "he" else 0.0 for kind in lay.kinds]
+    lr_mult = [0.5 if name.startswith("s3") else 1.0 for name in lay.names]
+    tables = [torch.empty(s.ctx.ssd_tensor_table_bytes(), dtype=torch.uint8, device="cuda") for s in (a, b)]
+    a.ctx.ssd_set_tensor_scales(lr_mult, wd_mult, tables[0])
+    b.ctx.ssd_set_tensor_scales(lr_mult, wd_mult, tables[1])
+    staging = [torch.empty(b.n, dtype=torch.float32, device="cuda") for _ in range(K)]
+    w_out = torch.empty(b.n, dtype=torch.float32).pin_memory()
+    chunks = -(-b.n // (1 << 24))
+    assert chunks == 2
+    for n in range(5):
+        grads = [synth.gradient(lay, n, i, 1e-3, device="cuda") for i in range(K)]
+        host = [g.cpu().pin_memory() for g in grads]
+        a.ctx.ssd_step(grads)
+        b.ctx.ssd_step_host(host, staging, w_out)
+        torch.cuda.synchronize()
+        assert torch.equal(w_out.view(torch.int32), a.w.cpu().view(torch.int32)), f"w_out iter {n}"
+    for name in ("w", "mom"):
+        assert torch.equal(getattr(a, name).view(torch.int32), getattr(b, name).view(torch.int32)), name
+    for i in range(K):
+        for name in ("w_loc", "pre", "w_dev"):
+            assert torch.equal(getattr(a, name)[i].view(torch.int32), getattr(b, name)[i].view(torch.int32)), name
+    assert b.ctx.ssd_kernel_launches() == 5 * chunks and a.ctx.ssd_get_counters()[:2] == b.ctx.ssd_get_counters()[:2]
