@@ -43,12 +43,11 @@ WORKLOADS = {
 }
 DEFAULT_WORKLOAD = "vgg16_K16"
 
-# DRAM bytes per parameter of one step_kernel launch (dram__bytes_read.sum + dram__bytes_write.sum
-# from an ncu capture on a flat arena of 2^24 parameters with the same worker count, gradient type
-# and launch shape; the kernel streams, so traffic grows in proportion to N), by iteration flags.
-# Valid only for the kernel sources with this digest.
-NCU_TRAFFIC = {"digest": "53dc9cc50d92e453", "K": 16, "grad_dtype": "f32",
-               "bytes_per_param": {0: 269.98, 2: 332.63, 4: 332.85}}
+# DRAM bytes per launch of step_kernel on the default workload (dram__bytes_read.sum +
+# dram__bytes_write.sum, one-pass ncu capture of this benchmark's own launches), by iteration flags
+# (0 plain, 2 refresh, 4 pull).  Valid only for the kernel sources with this digest.
+NCU_TRAFFIC = {"digest": "3b9a6f24297172c3", "workload": "vgg16_K16",
+               "bytes_per_launch": {0: 37599490816, 2: 46439410688, 4: 46441101056}}
 
 
 def kernel_digest() -> str:
@@ -318,10 +317,11 @@ def main():
     peak, peak_kind = measured_peak()
     achieved = (sum(bytes_per_launch) / len(bytes_per_launch)) / (statistics.mean(per_launch_ms) * 1e-3) / 1e9
     traffic = None
-    if NCU_TRAFFIC["digest"] == kernel_digest() and NCU_TRAFFIC["K"] == K and sg == 4 and not args.shared_pre:
-        per = NCU_TRAFFIC["bytes_per_param"]
+    if (NCU_TRAFFIC["digest"] == kernel_digest() and NCU_TRAFFIC["workload"] == wl_name
+            and not args.shared_pre and not args.per_tensor and not args.threads and not args.blocks_per_sm):
+        per = NCU_TRAFFIC["bytes_per_launch"]
         if all((f & 6) in per for f in flags_of):
-            traffic = N * statistics.mean(per[f & 6] for f in flags_of)
+            traffic = statistics.mean(per[f & 6] for f in flags_of)
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
