@@ -20,7 +20,13 @@ def bits(a):
 
 
 def assert_same(got, want, what, idx=None):
-    g = got.detach().cpu().numpy() if isinstance(got, torch.Tensor) else got
+    if isinstance(got, torch.Tensor):
+        if idx is not None:                       # gather on the device: the arena may be GiB-sized
+            got = got[torch.from_numpy(np.asarray(idx)).to(got.device)]
+            idx = None
+        g = got.detach().cpu().numpy()
+    else:
+        g = got
     if idx is not None:
         g = g[idx]
     gb, wb = bits(g), bits(want)

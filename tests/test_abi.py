@@ -234,3 +234,14 @@ def test_tensor_table_size_and_validation():
             ctx.ssd_set_tensor_scales(lr_mult, wd_mult, tbl)
         assert e.value.status == status
     ctx.ssd_set_tensor_scales(None, None, None)                  # uniform: nothing to upload
+
+
+def test_header_is_valid_c_and_cpp(tmp_path):
+    import subprocess
+    header = os.path.join(ROOT, "include", "ssd_sgd.h")
+    c = tmp_path / "use.c"
+    c.write_text('#include "ssd_sgd.h"\nint main(void) { ssd_hparams hp; hp.K = 1; return (int)sizeof(ssd_buffers) * 0 + hp.K - 1; }\n')
+    subprocess.check_call(["gcc", "-std=c99", "-pedantic", "-Wall", "-Werror", "-I", os.path.dirname(header),
+                           "-c", str(c), "-o", str(tmp_path / "use_c.o")])
+    subprocess.check_call(["g++", "-std=c++11", "-Wall", "-Werror", "-I", os.path.dirname(header), "-x", "c++",
+                           "-c", str(c), "-o", str(tmp_path / "use_cpp.o")])

@@ -99,47 +99,48 @@ def test_config_vgg16_K16_sampled():
     run_sampled("vgg16", 16, 4, 4, 20, 1e-3, 0.01, 0.9)
 
 
-def prime(n, K, bf16, device, idx=None):
-    """uniform(-1,1) state and gradients of the bandwidth sweep; at `idx` only when given."""
-    def buf(stream, worker=0):
-        if idx is None:
-            return synth.uniform_buffer(stream, n, worker=worker, device=device)
-        return synth.uniform_at(synth.stream_key(synth.SEED, stream, 0, worker), idx)
-    d = dict(w=buf(synth.STREAM_WEIGHT), mom=buf(synth.STREAM_MOM),
-             w_loc=[buf(synth.STREAM_WLOC, i) for i in range(K)],
-             pre=[buf(synth.STREAM_PRE, i) for i in range(K)],
-             g=[buf(synth.STREAM_GRAD, i) for i in range(K)])
-    if bf16:
-        d["g"] = [synth.to_bf16(g) for g in d["g"]]
-    return d
+def sweep_buffer(stream, n, worker, device, idx=None):
+    """One uniform(-1,1) buffer of the bandwidth sweep; only its elements at `idx` when given."""
+    if idx is None:
+        return synth.uniform_buffer(stream, n, worker=worker, device=device)
+    return synth.uniform_at(synth.stream_key(synth.SEED, stream, 0, worker), idx)
 
 
 def sweep_point(n, K, bf16, glu_flags, sampled):
+    """One server update, then one GLU update per worker, from primed uniform(-1,1) state."""
     ohp, chp = make_hp(K, 0.1, 0.9, 0, 4, bf16=bf16)
-    idx = None
+    idx = tidx = None
     if sampled:
         idx = np.unique(np.concatenate([np.arange(64), np.arange(n - 64, n),
                                         np.random.default_rng(n + K).integers(0, n, 4096)])).astype(np.int64)
-    d = prime(n, K, bf16, "cuda")
-    dev = DeviceState([n], chp, d["w"])
-    dev.mom.copy_(d["mom"])
+        tidx = torch.from_numpy(idx)
+
+    def host(stream, worker=0):
+        """The oracle's copy of a buffer: the sampled elements, or all of them."""
+        return sweep_buffer(stream, n, worker, "cpu", tidx).numpy().copy()
+
+    # the device state is filled in place, one buffer at a time (the largest points nearly fill the GPU)
+    dev = DeviceState([n], chp, sweep_buffer(synth.STREAM_WEIGHT, n, 0, "cuda"))
+    dev.mom.copy_(sweep_buffer(synth.STREAM_MOM, n, 0, "cuda"))
+    grads = []
     for i in range(K):
-        dev.w_loc[i].copy_(d["w_loc"][i]); dev.pre[i].copy_(d["pre"][i])
-    h = prime(n, K, bf16, "cpu", None if idx is None else torch.from_numpy(idx)) if sampled else None
-    def host(name, i=None):
-        t = (h if sampled else d)[name]
-        t = t if i is None else t[i]
-        return oracle_grad(t, bf16) if name == "g" else t.cpu().numpy().copy()
-    ref = oracle.State(ohp, host("w"))
-    ref.mom[:] = host("mom")
+        dev.w_loc[i].copy_(sweep_buffer(synth.STREAM_WLOC, n, i, "cuda"))
+        dev.pre[i].copy_(sweep_buffer(synth.STREAM_PRE, n, i, "cuda"))
+        g = sweep_buffer(synth.STREAM_GRAD, n, i, "cuda")
+        grads.append(synth.to_bf16(g) if bf16 else g)
+    ref = oracle.State(ohp, host(synth.STREAM_WEIGHT))
+    ref.mom[:] = host(synth.STREAM_MOM)
+    ref_grads = []
     for i in range(K):
-        ref.w_loc[i][:] = host("w_loc", i); ref.pre[i][:] = host("pre", i)
-    # one synchronous server update, then one GLU update per worker
-    dev.ctx.ssd_server_sync_update(d["g"])
-    oracle.server_update(ohp, [host("g", i) for i in range(K)], ref.w, ref.mom)
+        ref.w_loc[i][:] = host(synth.STREAM_WLOC, i)
+        ref.pre[i][:] = host(synth.STREAM_PRE, i)
+        g = sweep_buffer(synth.STREAM_GRAD, n, i, "cpu", tidx)
+        ref_grads.append(oracle_grad(synth.to_bf16(g) if bf16 else g, bf16))
+    dev.ctx.ssd_server_sync_update(grads)
+    oracle.server_update(ohp, ref_grads, ref.w, ref.mom)
     for i in range(K):
-        dev.ctx.ssd_worker_glu_update(i, d["g"][i], glu_flags)
-        oracle.glu_update(ohp, host("g", i), ref.w_loc[i], ref.pre[i], ref.w_dev[i], ref.w, glu_flags)
+        dev.ctx.ssd_worker_glu_update(i, grads[i], glu_flags)
+        oracle.glu_update(ohp, ref_grads[i], ref.w_loc[i], ref.pre[i], ref.w_dev[i], ref.w, glu_flags)
     torch.cuda.synchronize()
     tag = f"sweep n={n} K={K} bf16={bf16} flags={glu_flags}"
     assert_same(dev.w, ref.w, tag + " w", idx)
@@ -166,7 +167,8 @@ def test_sweep_refresh_and_pull_variants(bf16):
 @pytest.mark.parametrize("K,bf16", [(4, False), (32, True), (32, False)])
 def test_sweep_largest_size_sampled(K, bf16):
     n = 1 << 28
-    need = ((2 + 3 * K) * 4 + K * (2 if bf16 else 4)) * n * 1.1 + (4 << 30)
+    torch.cuda.empty_cache()
+    need = ((2 + 4 * K) * 4 + K * (2 if bf16 else 4)) * n + (8 << 30)      # state, gradients, generator scratch
     if torch.cuda.mem_get_info()[0] < need:
         pytest.skip(f"needs {need / 2**30:.0f} GiB of free device memory")
     sweep_point(n, K, bf16, 0, sampled=True)

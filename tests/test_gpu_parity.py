@@ -368,3 +368,28 @@ def test_shared_pre_weight_gives_the_same_results(bf16):
     with pytest.raises(B.SsdError) as e:
         dev.ctx.ssd_worker_local_step(0, grads[0])
     assert e.value.status == B.SSD_ERR_STATE
+
+
+def test_layout_with_empty_tensors_and_per_tensor_scales():
+    # zero-length tensors occupy no arena space; per-tensor lookups must skip them on both sides
+    K = 2
+    lay = synth.Layout("t")
+    for n in (0, 5, 0, 0, 9, 16, 0):
+        lay.add("x", n, "he", 4)
+    assert lay.padded_numel == 8 + 12 + 16
+    lr_mult = [9.0, 1.0, 9.0, 9.0, 0.5, 2.0, 9.0]
+    wd_mult = [9.0, 0.0, 9.0, 9.0, 1.0, 2.0, 9.0]
+    ohp, chp = make_hp(K, 0.1, 0.9, 1, 2, wd=0.01)
+    ohp.set_tensor_scales(tensor_ends(lay), lr_mult, wd_mult)
+    w0 = synth.init_weights(lay)
+    dev = DeviceState(lay.numels, chp, w0)
+    assert [dev.ctx.ssd_tensor_offset(t) for t in range(7)] == lay.offsets == [0, 0, 8, 8, 8, 20, 36]
+    table = torch.empty(dev.ctx.ssd_tensor_table_bytes(), dtype=torch.uint8, device="cuda")
+    dev.ctx.ssd_set_tensor_scales(lr_mult, wd_mult, table)
+    ref = oracle.State(ohp, w0.numpy())
+    for n in range(7):
+        grads = [synth.gradient(lay, n, i, 0.05, device="cuda") for i in range(K)]
+        dev.ctx.ssd_step(grads)
+        ref.step([oracle_grad(g, False) for g in grads])
+    torch.cuda.synchronize()
+    compare_states(dev, ref, "empty tensors")
