@@ -28,7 +28,10 @@
  *    NULL = the legacy default stream) and return; they never synchronise.
  *    Work of successive calls on the same stream is ordered by the stream.
  *  - Every call returns an ssd_status.  Arguments are validated before any
- *    launch; on an error nothing was enqueued and no counter moved.
+ *    launch: on an argument, alignment, layout or state error nothing was
+ *    enqueued and no counter moved.  SSD_ERR_CUDA reports a failure of the CUDA
+ *    runtime itself (ssd_last_cuda_error has its text); no counter moved, but
+ *    work enqueued before the failing call stays enqueued.
  *  - A context is not thread-safe; use one per host thread or lock around it.
  *
  * Arena layout.  A parameter layout is an ordered list of T tensors given by

@@ -393,3 +393,22 @@ def test_layout_with_empty_tensors_and_per_tensor_scales():
         ref.step([oracle_grad(g, False) for g in grads])
     torch.cuda.synchronize()
     compare_states(dev, ref, "empty tensors")
+
+
+def test_plain_c_program_reproduces_the_hand_trace(tmp_path):
+    # the boundary is usable from plain C: compile a C program against include/ssd_sgd.h, link it
+    # with the library and the CUDA runtime, run it
+    import os
+    import subprocess
+    from paper_2012_05396_b200 import build as libbuild
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    lib = libbuild.build_library()
+    cuda = os.environ.get("CUDA_HOME", "/usr/local/cuda")
+    exe = str(tmp_path / "trace_demo")
+    subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Werror", "-I", os.path.join(root, "include"),
+                           "-I", os.path.join(cuda, "include"), os.path.join(root, "tests", "c_abi", "trace_demo.c"),
+                           lib, "-L", os.path.join(cuda, "lib64"), "-lcudart", "-o", exe,
+                           "-Wl,-rpath," + os.path.dirname(lib), "-Wl,-rpath," + os.path.join(cuda, "lib64")])
+    r = subprocess.run([exe], capture_output=True, text=True, timeout=120)
+    assert r.returncode == 0, r.stdout + r.stderr
+    assert "trace reproduced from C" in r.stdout
