@@ -116,8 +116,17 @@ def _ptr(x) -> Optional[int]:
     return int(x)
 
 
-def _ptr_table(xs: Sequence):
+def _ptr_table(xs):
+    if isinstance(xs, C.Array):            # already marshalled by pointer_table()
+        return xs
     return (C.c_void_p * len(xs))(*[_ptr(x) for x in xs])
+
+
+def pointer_table(tensors: Sequence):
+    """Marshals a list of tensors / addresses once; the result can be passed wherever a list of
+    gradient or staging buffers is expected, which saves the per-call conversion when the same
+    buffers are used for many steps.  The caller keeps the tensors alive."""
+    return _ptr_table(list(tensors))
 
 
 def _stream(stream) -> Optional[int]:

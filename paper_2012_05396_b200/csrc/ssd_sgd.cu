@@ -6,9 +6,11 @@
 
 #include <cmath>
 #include <cstring>
+#include <map>
 #include <mutex>
 #include <new>
 #include <string>
+#include <utility>
 #include <vector>
 
 namespace {
@@ -16,6 +18,7 @@ namespace {
 using namespace ssd;
 
 constexpr int64_t kMaxArena = int64_t(1) << 40;
+constexpr int64_t kL2ResidentBytes = 128 << 20;         // a step moving less than this stays within the 126 MB L2
 constexpr int64_t kHostChunkElems = int64_t(1) << 24;   // ssd_step_host: elements per pipelined chunk
 
 struct Device {
@@ -46,6 +49,7 @@ struct ssd_ctx {
     // ssd_step_host pipelines chunks over two side streams (copies in, copies out)
     cudaStream_t in_stream = nullptr, out_stream = nullptr;
     std::vector<cudaEvent_t> events;
+    std::map<std::pair<const void *, int>, int> occupancy;   // (kernel, threads) -> blocks that fit per SM
     int64_t launches = 0;
     Device dev;
     std::string cuda_error;
@@ -129,10 +133,18 @@ struct Shape {
 template <typename Kernel>
 ssd_status grid_for(ssd_ctx *c, Kernel kernel, int64_t n, const Shape &sh, int *grid)
 {
+    // resident blocks per SM of this kernel at this block size: asked once, then remembered
+    const std::pair<const void *, int> key(reinterpret_cast<const void *>(kernel), sh.threads);
     int fit = 0;
-    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&fit, kernel, sh.threads, 0);
-    if (e != cudaSuccess) return cuda_fail(c, e);
-    if (fit < 1) fit = 1;
+    auto hit = c->occupancy.find(key);
+    if (hit != c->occupancy.end()) {
+        fit = hit->second;
+    } else {
+        cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&fit, kernel, sh.threads, 0);
+        if (e != cudaSuccess) return cuda_fail(c, e);
+        if (fit < 1) fit = 1;
+        c->occupancy[key] = fit;
+    }
     const int per_sm = (sh.per_sm > 0 && sh.per_sm < fit) ? sh.per_sm : fit;
     const int64_t nvec = n / sh.vw;
     int64_t need = (nvec + sh.threads - 1) / sh.threads;
@@ -207,7 +219,12 @@ Shape step_shape(const ssd_ctx *c, int flags, bool wide_ok)
     // Iterations that add K stores per element (pull; refresh or first call with one pre_weight
     // per worker) are write-heavy: 512 threads per SM.  The others: 640 threads per SM.
     const bool k_extra_stores = (flags & kPull) || (!c->shared_pre && (flags & (kRefresh | kFirst)));
-    const Shape sh = k_extra_stores ? Shape{8, 1, 128, 4} : Shape{8, 1, 128, 5};
+    Shape sh = k_extra_stores ? Shape{8, 1, 128, 4} : Shape{8, 1, 128, 5};
+    // A step whose whole traffic fits in L2 (ResNet-20/56 sized arenas) is bound by latency, not by
+    // DRAM: smaller vectors spread it over more threads, and two workers' loads per thread halve the
+    // number of dependent round trips.
+    const int64_t sg = c->hp.grad_dtype == SSD_BF16 ? 2 : 4;
+    if (c->n * (c->hp.K * (sg + 12) + 16) < kL2ResidentBytes) sh = Shape{4, 2, 64, 0};
     return finish_shape(c, sh, wide_ok, 4);
 }
 
