@@ -40,7 +40,8 @@ class _HP(C.Structure):
                 ("lr", C.c_float), ("m", C.c_float), ("wd", C.c_float),
                 ("lr_loc", C.c_float), ("alpha", C.c_float), ("beta", C.c_float),
                 ("rescale", C.c_float), ("T", C.c_int32), ("tensor_end", C.c_void_p),
-                ("lr_mult", C.c_void_p), ("wd_mult", C.c_void_p), ("arena_index", C.c_void_p)]
+                ("lr_mult", C.c_void_p), ("wd_mult", C.c_void_p), ("arena_index", C.c_void_p),
+                ("local_sgd", C.c_int32)]
 
 
 class _State(C.Structure):
@@ -97,8 +98,9 @@ class Hyper:
 
     def __init__(self, K: int, lr: float, m: float, W: int, k: int, wd: float = 0.0,
                  lr_loc: Optional[float] = None, alpha: float = 2.0, beta: float = 0.5,
-                 rescale: Optional[float] = None, grad_bf16: bool = False):
+                 rescale: Optional[float] = None, grad_bf16: bool = False, local_sgd: bool = False):
         f32 = np.float32
+        self.local_sgd = bool(local_sgd)        # workers update with plain SGD (Eq. 5) instead of GLU
         self.K, self.W, self.k = int(K), int(W), int(k)
         self.lr, self.m, self.wd = f32(lr), f32(m), f32(wd)
         self.lr_loc = f32(4.0) * f32(lr) if lr_loc is None else f32(lr_loc)
@@ -122,7 +124,7 @@ class Hyper:
         return _HP(self.K, int(self.grad_bf16), self.W, self.k, float(self.lr), float(self.m),
                    float(self.wd), float(self.lr_loc), float(self.alpha), float(self.beta),
                    float(self.rescale), T, ptr(self.tensor_end), ptr(self.lr_mult), ptr(self.wd_mult),
-                   ptr(self.arena_index))
+                   ptr(self.arena_index), int(self.local_sgd))
 
 
 def schedule(n: int, W: int, k: int):

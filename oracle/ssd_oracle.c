@@ -53,6 +53,10 @@ typedef struct {
     const float *wd_mult;        /* multiplies wd of tensor t                        */
     const int64_t *arena_index;  /* optional: arena position of local element j (for
                                     runs on a gathered sample of the arena)          */
+    /* Local updater of the workers (Section 4.4 compares them): 0 = GLU, 1 = plain SGD,
+     * i.e. Eq. 5 with the descent sign, w' = w' - lr_loc*(grad' + wd*w'): no grad_sync,
+     * pre_weight is neither read nor written, alpha and beta are not used. */
+    int32_t local_sgd;
 } oracle_hp;
 
 typedef struct {
@@ -177,6 +181,17 @@ void oracle_glu_update(int64_t N, const oracle_hp *hp, const void *g,
     for (int64_t j = 0; j < N; ++j) {
         const tensor_scalars ts = hp->T ? scalars_at(hp, j) : uniform;
         const real lr_loc = ts.lr_loc, wd = ts.wd, c = ts.c;
+        if (hp->local_sgd) {
+            real decay_l = wd * w_loc[j];
+            real full_l = grad_at(g, hp->grad_bf16, j) + decay_l;
+            real step_l = lr_loc * full_l;
+            w_loc[j] = w_loc[j] - step_l;
+            if (flags & F_PULL) {
+                w_dev[j] = w_loc[j];
+                w_loc[j] = w_server[j];
+            }
+            continue;
+        }
         if (flags & F_FIRST) pre[j] = w_loc[j];
         real diff = pre[j] - w_loc[j];
         real grad_sync = diff * c;

@@ -13,6 +13,7 @@ import pytest
 import oracle
 from tests import golden_trace
 from tests.test_oracle_pins import paper_counters, per_tensor_composition_holds
+from tests import test_oracle_pins
 
 SRC = os.path.join(os.path.dirname(oracle.__file__), "ssd_oracle.c")
 
@@ -40,6 +41,10 @@ MUTATIONS = [
     ("pull one iteration early", "d % k == k - 1", "(d + 1) % k == k - 1"),
     ("refresh on the first call", "if (d > 0 && d % k == 0)", "if (d % k == 0)"),
     ("warm-up off by one", "if (k == 0 || n < W)", "if (k == 0 || n <= W)"),
+    ("local SGD adds its step", "w_loc[j] = w_loc[j] - step_l;", "w_loc[j] = w_loc[j] + step_l;"),
+    ("local SGD forgets weight decay", "real decay_l = wd * w_loc[j];", "real decay_l = 0 * w_loc[j];"),
+    ("local SGD uses the server lr", "real step_l = lr_loc * full_l;", "real step_l = (real)hp->lr * full_l;"),
+    ("local SGD pull keeps the local result", "w_dev[j] = w_loc[j];\n                w_loc[j] = w_server[j];\n            }\n            continue;", "w_dev[j] = w_server[j];\n            }\n            continue;"),
     ("tensor lookup off by one", "pos >= hp->tensor_end[t]", "pos > hp->tensor_end[t]"),
     ("local lr ignores the tensor's multiplier", "float lr_loc_t = hp->lr_loc * hp->lr_mult[t];", "float lr_loc_t = hp->lr_loc;"),
     ("decay multiplier taken from lr_mult", "float wd_t = hp->wd * hp->wd_mult[t];", "float wd_t = hp->wd * hp->lr_mult[t];"),
@@ -90,7 +95,14 @@ def traces_pass(lib):
                 ref = paper_counters(W, k, W + 3 * k + 2)
                 if [oracle.schedule(n, W, k) for n in range(len(ref))] != ref:
                     return False
-        return per_tensor_composition_holds()
+        if not per_tensor_composition_holds():
+            return False
+        try:
+            test_oracle_pins.test_local_sgd_updater_is_eq5_and_never_touches_pre_weight()
+            test_oracle_pins.test_local_sgd_equals_glu_with_alpha_one_beta_zero()
+        except AssertionError:
+            return False
+        return True
     finally:
         if saved is not None:
             oracle._libs[False] = saved

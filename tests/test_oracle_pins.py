@@ -551,3 +551,44 @@ def test_server_trajectory_independent_of_schedule_with_multipliers_and_lr_chang
         st = run(W, k)
         np.testing.assert_array_equal(st.w, ref.w)
         np.testing.assert_array_equal(st.mom, ref.mom)
+
+
+# ---------------------------------------------------------------------------
+# plain SGD as the workers' local updater (Eq. 5; compared with GLU in Section 4.4)
+# ---------------------------------------------------------------------------
+
+def test_local_sgd_updater_is_eq5_and_never_touches_pre_weight():
+    rng = np.random.default_rng(14)
+    K, N, W, k, T = 3, 11, 2, 3, 12
+    w0 = rng.standard_normal(N).astype(f32)
+    stream = [rng_grads(rng, K, N, 0.1) for _ in range(T)]
+    hp = Hyper(K=K, lr=0.1, m=0.9, W=W, k=k, wd=0.01, lr_loc=0.25, local_sgd=True)
+    st = State(hp, w0, fill=123.0)
+    shadow = None                                  # Eq. 5 in double, worker 1
+    for n, gs in enumerate(stream):
+        before = st.w_loc[1].astype(np.float64)
+        stage, flags = st.step(gs)
+        if stage == STAGE_DELAY:
+            expect = before - 0.25 * (gs[1].astype(np.float64) + float(hp.wd) * before)
+            got = st.w_dev[1] if flags & F_PULL else st.w_loc[1]
+            np.testing.assert_allclose(got, expect, rtol=1e-6, atol=1e-7)
+            if flags & F_PULL:
+                np.testing.assert_array_equal(st.w_loc[1], st.w)
+    for i in range(K):
+        assert np.all(st.pre[i] == f32(123.0))      # no pre_weight in this updater
+    # and the server does not care which local updater the workers use
+    ref, _ = run_config(Hyper(K=K, lr=0.1, m=0.9, W=W, k=k, wd=0.01, lr_loc=0.25), w0, stream)
+    np.testing.assert_array_equal(st.w, ref.w)
+    np.testing.assert_array_equal(st.mom, ref.mom)
+
+
+def test_local_sgd_equals_glu_with_alpha_one_beta_zero():
+    rng = np.random.default_rng(15)
+    K, N, T = 2, 64, 10
+    w0 = rng.standard_normal(N).astype(f32)
+    stream = [rng_grads(rng, K, N, 0.1) for _ in range(T)]
+    a, _ = run_config(Hyper(K=K, lr=0.1, m=0.9, W=1, k=2, wd=0.01, lr_loc=0.3, local_sgd=True), w0, stream)
+    b, _ = run_config(Hyper(K=K, lr=0.1, m=0.9, W=1, k=2, wd=0.01, lr_loc=0.3, alpha=1.0, beta=0.0), w0, stream)
+    for i in range(K):
+        np.testing.assert_array_equal(a.w_loc[i], b.w_loc[i])
+        np.testing.assert_array_equal(a.w_dev[i], b.w_dev[i])
