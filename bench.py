@@ -58,11 +58,13 @@ def kernel_digest() -> str:
     return h.hexdigest()[:16]
 
 
-def step_bytes_per_param(K: int, sg: int, flags: int, shared_pre: bool = False) -> int:
+def step_bytes_per_param(K: int, sg: int, flags: int, shared_pre: bool = False, local_sgd: bool = False) -> int:
     """Algorithmic bytes one fused delay-stage step moves per parameter: K gradients, K local
     weights read and written, K pre_weights read, w and mom read and written; a refresh adds K
     pre_weight stores, a pull adds K device-weight stores (and trades nothing else).  With one
     shared pre_weight buffer it is read once and refreshed once instead of K times."""
+    if local_sgd:       # plain-SGD local updater: no pre_weight traffic at all
+        return K * (sg + 8) + 16 + (4 * K if flags & 4 else 0)
     pre_copies = 1 if shared_pre else K
     b = K * (sg + 8) + 4 * pre_copies + 16
     if flags & 2:       # refresh
@@ -228,6 +230,8 @@ def main():
                     help="per-tensor hyper-parameters: weight decay 5e-4 on conv/FC weights only")
     ap.add_argument("--shared-pre", action="store_true",
                     help="one pre_weight buffer shared by all workers (fewer algorithmic bytes, counted as such)")
+    ap.add_argument("--local-sgd", action="store_true",
+                    help="workers update with plain SGD (Eq. 5) instead of GLU (fewer algorithmic bytes, counted as such)")
     ap.add_argument("--threads", type=int, default=0, help="threads per block (0 = library default)")
     ap.add_argument("--blocks-per-sm", type=int, default=0, help="resident blocks per SM (0 = default)")
     args = ap.parse_args()
@@ -266,7 +270,8 @@ def main():
 
     nan = float("nan")
     hp = B.make_hparams(K, wl["lr"], wl["m"], wl["W"], wl["k"], wd=5e-4 if args.per_tensor else 0.0,
-                        lr_local=nan, alpha=nan, beta=nan, rescale=nan, grad_dtype=B.SSD_F32)
+                        lr_local=nan, alpha=nan, beta=nan, rescale=nan, grad_dtype=B.SSD_F32,
+                        local_updater=B.SSD_LOCAL_SGD if args.local_sgd else B.SSD_LOCAL_GLU)
     w0 = synth.init_weights(lay, device=dev_name)
     st = DeviceState(lay.numels, hp, w0, device=dev_name, fill=0.0, shared_pre=args.shared_pre)
     if args.per_tensor:
@@ -312,13 +317,13 @@ def main():
     total_ms = ev[0].elapsed_time(ev[-1])
     per_launch_ms = [ev[n].elapsed_time(ev[n + 1]) for n in range(args.steps)]
     total_ms = max_over_ranks(total_ms, dev_name, world)
-    bytes_per_launch = [step_bytes_per_param(K, sg, f, args.shared_pre) * N for f in flags_of]
+    bytes_per_launch = [step_bytes_per_param(K, sg, f, args.shared_pre, args.local_sgd) * N for f in flags_of]
     value = whole_job_rate(float(sum(bytes_per_launch)), world, total_ms) / 1e9
     peak, peak_kind = measured_peak()
     achieved = (sum(bytes_per_launch) / len(bytes_per_launch)) / (statistics.mean(per_launch_ms) * 1e-3) / 1e9
     traffic = None
     if (NCU_TRAFFIC["digest"] == kernel_digest() and NCU_TRAFFIC["workload"] == wl_name
-            and not args.shared_pre and not args.per_tensor and not args.threads and not args.blocks_per_sm):
+            and not args.shared_pre and not args.local_sgd and not args.per_tensor and not args.threads and not args.blocks_per_sm):
         per = NCU_TRAFFIC["bytes_per_launch"]
         if all((f & 6) in per for f in flags_of):
             traffic = statistics.mean(per[f & 6] for f in flags_of)
@@ -335,6 +340,7 @@ def main():
                    "stage": "steps-delay", "kernel": "fused ssd_step", "replicas": world,
                    "hyper_parameters": "per tensor" if args.per_tensor else "uniform",
                    "pre_weight": "one shared buffer" if args.shared_pre else "one buffer per worker",
+                   "local_updater": "sgd" if args.local_sgd else "glu",
                    "device_bytes": st.bytes() + n_sets * K * N * sg,
                    "l2": "inputs larger than L2 (no flush needed)"
                    if st.bytes() > 4 * 126e6 else "L2-resident: not an HBM measurement"},
@@ -369,7 +375,7 @@ def main():
         torch.cuda.synchronize()
         e_ms = e0.elapsed_time(e1)
         e_ms = max_over_ranks(e_ms, dev_name, world)
-        e_bytes = float(sum(step_bytes_per_param(K, sg, f, args.shared_pre) * N for f in e_flags))
+        e_bytes = float(sum(step_bytes_per_param(K, sg, f, args.shared_pre, args.local_sgd) * N for f in e_flags))
         e2e = {"value": whole_job_rate(e_bytes, world, e_ms) / 1e9, "unit": UNIT, "h2d_bytes_per_step": K * N * sg,
                "d2h_bytes_per_step": N * 4, "steps": args.e2e_steps, "ms_per_step": e_ms / args.e2e_steps,
                "call": "ssd_step_host"}

@@ -79,6 +79,13 @@ typedef enum {
 
 typedef enum { SSD_F32 = 0, SSD_BF16 = 1 } ssd_dtype;
 
+/* Local updater of the workers in the delay stage.  The paper's is GLU; its Section
+ * 4.4 compares it with plain SGD, Eq. 5 (with the descent sign):
+ *     w_loc_i[j] = w_loc_i[j] - lr_local * (g_i[j] + wd * w_loc_i[j])
+ * which has no grad_sync: pre_weight is neither read nor written (the FIRST and
+ * REFRESH flags have no effect) and alpha and beta are not used.  Pulls work the same. */
+typedef enum { SSD_LOCAL_GLU = 0, SSD_LOCAL_SGD = 1 } ssd_local_updater;
+
 enum { SSD_STAGE_WARMUP = 0, SSD_STAGE_DELAY = 1 };
 enum { SSD_FLAG_FIRST = 1, SSD_FLAG_REFRESH = 2, SSD_FLAG_PULL = 4, SSD_FLAG_COPY = 8 };
 enum { SSD_VIEW_GLOBAL = 0, SSD_VIEW_LOCAL = 1, SSD_VIEW_DEVICE = 2 };
@@ -104,6 +111,7 @@ typedef struct {
     float beta;                   /* weight of grad_sync; NaN = 0.5             */
     float rescale;                /* factor on the K-sum; NaN = 1/K (average)   */
     int32_t grad_dtype;           /* ssd_dtype of every gradient buffer         */
+    int32_t local_updater;        /* ssd_local_updater; 0 = GLU                  */
 } ssd_hparams;
 
 /* Caller-owned device state.  w_loc, pre, w_dev: host arrays of K device pointers.

@@ -22,6 +22,7 @@ LIB_PATH = os.environ.get("SSD_SGD_LIBRARY") or os.path.join(_HERE, "libssd_sgd.
  SSD_ERR_TOO_LARGE) = range(8)
 SSD_STATIC_TABLE_MAX_TENSORS = 1024
 SSD_F32, SSD_BF16 = 0, 1
+SSD_LOCAL_GLU, SSD_LOCAL_SGD = 0, 1
 SSD_STAGE_WARMUP, SSD_STAGE_DELAY = 0, 1
 SSD_FLAG_FIRST, SSD_FLAG_REFRESH, SSD_FLAG_PULL, SSD_FLAG_COPY = 1, 2, 4, 8
 SSD_VIEW_GLOBAL, SSD_VIEW_LOCAL, SSD_VIEW_DEVICE = 0, 1, 2
@@ -45,7 +46,7 @@ class ssd_hparams(C.Structure):
     _fields_ = [("K", C.c_int32), ("lr", C.c_float), ("momentum", C.c_float), ("wd", C.c_float),
                 ("warmup_iters", C.c_int32), ("delay_k", C.c_int32), ("lr_local", C.c_float),
                 ("alpha", C.c_float), ("beta", C.c_float), ("rescale", C.c_float),
-                ("grad_dtype", C.c_int32)]
+                ("grad_dtype", C.c_int32), ("local_updater", C.c_int32)]
 
 
 class ssd_buffers(C.Structure):
@@ -153,9 +154,10 @@ def ssd_arena_numel(numels: Sequence[int]) -> int:
 
 def make_hparams(K: int, lr: float, momentum: float, warmup_iters: int, delay_k: int, wd: float = 0.0,
                  lr_local: float = math.nan, alpha: float = math.nan, beta: float = math.nan,
-                 rescale: float = math.nan, grad_dtype: int = SSD_F32) -> ssd_hparams:
+                 rescale: float = math.nan, grad_dtype: int = SSD_F32,
+                 local_updater: int = SSD_LOCAL_GLU) -> ssd_hparams:
     return ssd_hparams(K, lr, momentum, wd, warmup_iters, delay_k, lr_local, alpha, beta, rescale,
-                       grad_dtype)
+                       grad_dtype, local_updater)
 
 
 class Context:

@@ -37,7 +37,7 @@ namespace ssd {
 constexpr int kMaxWorkers = 32;
 constexpr int kMaxThreads = 512;   // upper bound of threads per block for every kernel here
 
-enum : int { kFirst = 1, kRefresh = 2, kPull = 4, kCopy = 8 };
+enum : int { kFirst = 1, kRefresh = 2, kPull = 4, kCopy = 8, kLocalSgd = 16 };   // kLocalSgd: internal
 enum : int { kF32 = 0, kBF16 = 1 };
 
 struct Scalars {
@@ -213,6 +213,12 @@ __device__ __forceinline__ float glu_elem(float g, float wl, float pre, const Sc
     return __fsub_rn(wl, __fmul_rn(s.lr_loc, mix));
 }
 
+// Plain SGD as local updater (Eq. 5 with the descent sign): w' - lr_loc*(g + wd*w').
+__device__ __forceinline__ float local_sgd_elem(float g, float wl, const Scalars &s)
+{
+    return __fsub_rn(wl, __fmul_rn(s.lr_loc, __fadd_rn(g, __fmul_rn(s.wd, wl))));
+}
+
 // ---------------------------------------------------------------------------
 // Per-tensor scalars.  Tensors start on multiples of 4 elements, so each group of
 // 4 consecutive elements lies in one tensor; a vector of 8 may straddle two.  The
@@ -290,16 +296,18 @@ __device__ __forceinline__ void sync_at(const SyncParams &p, int64_t e)
 template <int GT, int VW, bool PT>
 __device__ __forceinline__ void glu_at(const GluParams &p, int64_t e)
 {
-    const bool first = p.flags & kFirst, refresh = p.flags & kRefresh, pull = p.flags & kPull;
+    const bool sgd = p.flags & kLocalSgd;      // plain-SGD updater: pre_weight is not involved at all
+    const bool first = (p.flags & kFirst) && !sgd, refresh = (p.flags & kRefresh) && !sgd, pull = p.flags & kPull;
     Grad<GT, VW> g = ld_grad<GT, VW>(p.g, e);
     Vec<VW> wl = ld_f32<VW>(p.w_loc, e);
-    Vec<VW> pr = first ? wl : ld_f32<VW>(p.pre, e);
+    Vec<VW> pr = (first || sgd) ? wl : ld_f32<VW>(p.pre, e);
     Vec<VW> wg;
     if (pull) wg = ld_f32<VW>(p.w, e);
     Vec<VW> r;
     const GroupScalars<PT, VW> sc(p.s, p.tt, e);
 #pragma unroll
-    for (int l = 0; l < VW; ++l) r.v[l] = glu_elem(g.get(l), wl.v[l], pr.v[l], sc.at(l));
+    for (int l = 0; l < VW; ++l)
+        r.v[l] = sgd ? local_sgd_elem(g.get(l), wl.v[l], sc.at(l)) : glu_elem(g.get(l), wl.v[l], pr.v[l], sc.at(l));
     if (first || refresh) st_f32<VW>(p.pre, e, wl);
     if (pull) {
         st_f32<VW>(p.w_dev, e, r);
@@ -312,7 +320,8 @@ __device__ __forceinline__ void glu_at(const GluParams &p, int64_t e)
 template <int GT, int VW, int B, bool PT>
 __device__ __forceinline__ void step_at(const StepParams &p, int64_t e)
 {
-    const bool first = p.flags & kFirst, refresh = p.flags & kRefresh, pull = p.flags & kPull;
+    const bool sgd = p.flags & kLocalSgd;      // plain-SGD updater: pre_weight is not involved at all
+    const bool first = (p.flags & kFirst) && !sgd, refresh = (p.flags & kRefresh) && !sgd, pull = p.flags & kPull;
     Vec<VW> w = ld_f32<VW>(p.w, e);
     Vec<VW> mom = ld_f32<VW>(p.mom, e);
     Vec<VW> sum;
@@ -321,7 +330,7 @@ __device__ __forceinline__ void step_at(const StepParams &p, int64_t e)
     // global weight, so worker 0's value is everyone's.
     const bool shared = p.shared_pre != 0;
     Vec<VW> pre_shared;
-    if (shared && !first) pre_shared = ld_f32<VW>(p.pre[0], e);
+    if (shared && !first && !sgd) pre_shared = ld_f32<VW>(p.pre[0], e);
     GroupScalars<PT, VW> sc(p.s, p.tt, e);
     for (int i0 = 0; i0 < p.K; i0 += B) {
         Grad<GT, VW> g[B];
@@ -331,7 +340,7 @@ __device__ __forceinline__ void step_at(const StepParams &p, int64_t e)
             if (i0 + b < p.K) {
                 g[b] = ld_grad<GT, VW>(p.g[i0 + b], e);
                 wl[b] = ld_f32<VW>(p.w_loc[i0 + b], e);
-                if (!first && !shared) pr[b] = ld_f32<VW>(p.pre[i0 + b], e);
+                if (!first && !shared && !sgd) pr[b] = ld_f32<VW>(p.pre[i0 + b], e);
             }
         }
 #pragma unroll
@@ -343,8 +352,8 @@ __device__ __forceinline__ void step_at(const StepParams &p, int64_t e)
                 for (int l = 0; l < VW; ++l) {
                     const float gl = g[b].get(l);
                     sum.v[l] = (i == 0) ? gl : __fadd_rn(sum.v[l], gl);
-                    const float pl = first ? wl[b].v[l] : shared ? pre_shared.v[l] : pr[b].v[l];
-                    r.v[l] = glu_elem(gl, wl[b].v[l], pl, sc.at(l));
+                    const float pl = (first || sgd) ? wl[b].v[l] : shared ? pre_shared.v[l] : pr[b].v[l];
+                    r.v[l] = sgd ? local_sgd_elem(gl, wl[b].v[l], sc.at(l)) : glu_elem(gl, wl[b].v[l], pl, sc.at(l));
                 }
                 if ((first || refresh) && (!shared || i == 0)) st_f32<VW>(p.pre[i], e, wl[b]);
                 st_f32<VW>(pull ? p.w_dev[i] : p.w_loc[i], e, r);

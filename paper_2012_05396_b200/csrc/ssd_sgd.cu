@@ -218,7 +218,8 @@ Shape step_shape(const ssd_ctx *c, int flags, bool wide_ok)
 {
     // Iterations that add K stores per element (pull; refresh or first call with one pre_weight
     // per worker) are write-heavy: 512 threads per SM.  The others: 640 threads per SM.
-    const bool k_extra_stores = (flags & kPull) || (!c->shared_pre && (flags & (kRefresh | kFirst)));
+    const bool sgd = c->hp.local_updater == SSD_LOCAL_SGD;
+    const bool k_extra_stores = (flags & kPull) || (!c->shared_pre && !sgd && (flags & (kRefresh | kFirst)));
     Shape sh = k_extra_stores ? Shape{8, 1, 128, 4} : Shape{8, 1, 128, 5};
     // A step whose whole traffic fits in L2 (ResNet-20/56 sized arenas) is bound by latency, not by
     // DRAM: smaller vectors spread it over more threads, and two workers' loads per thread halve the
@@ -349,7 +350,7 @@ ssd_status launch_glu(ssd_ctx *c, int worker, const void *grad, int flags, cudaS
     p.w_dev = c->w_dev[worker];
     p.w = c->w;
     p.n = c->n;
-    p.flags = flags;
+    p.flags = flags | (c->hp.local_updater == SSD_LOCAL_SGD ? kLocalSgd : 0);
     p.s = c->s;
     p.tt = table_of(c);
     const Shape sh = glu_shape(c, can_use_256bit(c, c->state32, &grad, 1));
@@ -389,7 +390,7 @@ ssd_status launch_step(ssd_ctx *c, const void *const *grads, int flags, cudaStre
     p.mom = c->mom + lo;
     p.n = count < 0 ? c->n : count;
     p.K = c->hp.K;
-    p.flags = flags;
+    p.flags = flags | (c->hp.local_updater == SSD_LOCAL_SGD ? kLocalSgd : 0);
     p.shared_pre = c->shared_pre ? 1 : 0;
     p.s = c->s;
     p.tt = table_of(c);
@@ -473,6 +474,7 @@ ssd_status ssd_init(ssd_ctx **out, const ssd_layout *layout, const ssd_hparams *
     if (!std::isfinite(hp->wd)) return SSD_ERR_ARG;
     if (hp->warmup_iters < 0 || hp->delay_k < 0) return SSD_ERR_ARG;
     if (hp->grad_dtype != SSD_F32 && hp->grad_dtype != SSD_BF16) return SSD_ERR_ARG;
+    if (hp->local_updater != SSD_LOCAL_GLU && hp->local_updater != SSD_LOCAL_SGD) return SSD_ERR_ARG;
     if (std::isinf(hp->lr_local) || std::isinf(hp->alpha) || std::isinf(hp->beta) ||
         std::isinf(hp->rescale))
         return SSD_ERR_ARG;

@@ -49,7 +49,7 @@ int main(void)
 
     const int64_t numel[1] = {N};
     ssd_layout layout = {1, numel};
-    ssd_hparams hp = {K, 0.5f, 0.5f, 0.0f, 1, 2, 2.0f, 2.0f, 0.5f, 0.5f, SSD_F32};
+    ssd_hparams hp = {K, 0.5f, 0.5f, 0.0f, 1, 2, 2.0f, 2.0f, 0.5f, 0.5f, SSD_F32, SSD_LOCAL_GLU};
     ssd_buffers bufs = {w, mom, w_loc, pre, w_dev};
     ssd_ctx *ctx = NULL;
     int64_t padded = 0;

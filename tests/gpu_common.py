@@ -40,14 +40,16 @@ def assert_same(got, want, what, idx=None):
     assert np.all(err <= ABS_TOL + REL_TOL * np.abs(want[finite].astype(np.float64))), what
 
 
-def make_hp(K, lr, m, W, k, wd=0.0, lr_loc=None, alpha=2.0, beta=0.5, rescale=None, bf16=False):
+def make_hp(K, lr, m, W, k, wd=0.0, lr_loc=None, alpha=2.0, beta=0.5, rescale=None, bf16=False,
+            local_sgd=False):
     """The same hyper-parameters for both sides (defaults resolved by each side on its own)."""
     nan = float("nan")
     o = oracle.Hyper(K=K, lr=lr, m=m, W=W, k=k, wd=wd, lr_loc=lr_loc, alpha=alpha, beta=beta,
-                     rescale=rescale, grad_bf16=bf16)
+                     rescale=rescale, grad_bf16=bf16, local_sgd=local_sgd)
     c = B.make_hparams(K, lr, m, W, k, wd=wd, lr_local=nan if lr_loc is None else lr_loc,
                        alpha=alpha, beta=beta, rescale=nan if rescale is None else rescale,
-                       grad_dtype=B.SSD_BF16 if bf16 else B.SSD_F32)
+                       grad_dtype=B.SSD_BF16 if bf16 else B.SSD_F32,
+                       local_updater=B.SSD_LOCAL_SGD if local_sgd else B.SSD_LOCAL_GLU)
     return o, c
 
 

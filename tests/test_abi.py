@@ -74,7 +74,7 @@ def test_layout_offsets_match_the_generator_module():
     ("lr", -1.0, B.SSD_ERR_ARG), ("lr", math.inf, B.SSD_ERR_ARG), ("lr", math.nan, B.SSD_ERR_ARG),
     ("momentum", 1.0, B.SSD_ERR_ARG), ("momentum", -0.1, B.SSD_ERR_ARG),
     ("wd", math.nan, B.SSD_ERR_ARG), ("warmup_iters", -1, B.SSD_ERR_ARG), ("delay_k", -1, B.SSD_ERR_ARG),
-    ("grad_dtype", 2, B.SSD_ERR_ARG), ("alpha", math.inf, B.SSD_ERR_ARG),
+    ("grad_dtype", 2, B.SSD_ERR_ARG), ("alpha", math.inf, B.SSD_ERR_ARG), ("local_updater", 2, B.SSD_ERR_ARG),
 ])
 def test_init_rejects_bad_hyper_parameters(field, value, status):
     K = 4

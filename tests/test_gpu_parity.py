@@ -412,3 +412,23 @@ def test_plain_c_program_reproduces_the_hand_trace(tmp_path):
     r = subprocess.run([exe], capture_output=True, text=True, timeout=120)
     assert r.returncode == 0, r.stdout + r.stderr
     assert "trace reproduced from C" in r.stdout
+
+
+@pytest.mark.parametrize("mode", ["fused", "split"])
+@pytest.mark.parametrize("bf16", [False, True])
+def test_plain_sgd_local_updater(mode, bf16):
+    # Eq. 5 as the workers' updater: no grad_sync, pre_weight never read or written
+    K, W, k, iters = 3, 2, 3, 11
+    lay = synth.get_layout("resnet20")
+    ohp, chp = make_hp(K, 0.1, 0.9, W, k, wd=1e-3, lr_loc=0.25, bf16=bf16, local_sgd=True)
+    w0 = synth.init_weights(lay)
+    dev = DeviceState(lay.numels, chp, w0)
+    ref = oracle.State(ohp, w0.numpy())
+    for n in range(iters):
+        grads = [synth.gradient(lay, n, i, 1e-2, device="cuda") for i in range(K)]
+        if bf16:
+            grads = [synth.to_bf16(g) for g in grads]
+        gpu_iteration(dev, grads, mode)
+        ref.step([oracle_grad(g, bf16) for g in grads])
+    torch.cuda.synchronize()
+    compare_states(dev, ref, "local SGD")                   # pre stays at its NaN fill on both sides
