@@ -432,3 +432,34 @@ def test_plain_sgd_local_updater(mode, bf16):
         ref.step([oracle_grad(g, bf16) for g in grads])
     torch.cuda.synchronize()
     compare_states(dev, ref, "local SGD")                   # pre stays at its NaN fill on both sides
+
+
+def test_work_is_ordered_on_the_callers_stream():
+    # everything is enqueued on the stream it is given: a side stream, with the gradients produced on
+    # that stream right before each call and no host synchronisation in between
+    K, W, k, iters = 4, 1, 2, 9
+    lay = synth.get_layout("resnet56")
+    ohp, chp = make_hp(K, 0.1, 0.9, W, k)
+    w0 = synth.init_weights(lay)
+    dev = DeviceState(lay.numels, chp, w0)
+    ref = oracle.State(ohp, w0.numpy())
+    side = torch.cuda.Stream()
+    staging = [torch.empty(dev.n, dtype=torch.float32, device="cuda") for _ in range(K)]
+    w_out = torch.empty(dev.n, dtype=torch.float32).pin_memory()
+    torch.cuda.synchronize()
+    kept = []
+    with torch.cuda.stream(side):
+        for n in range(iters):
+            grads = [synth.gradient(lay, n, i, 1e-2, device="cuda") for i in range(K)]
+            kept.append(grads)
+            if n % 3 == 2:                                  # mix in the host-gradient entry point
+                host = [g.cpu().pin_memory() for g in grads]
+                dev.ctx.ssd_step_host(host, staging, w_out, stream=side)
+                kept.append(host)
+            else:
+                dev.ctx.ssd_step(grads, stream=side)
+    side.synchronize()
+    for n in range(iters):
+        ref.step([synth.gradient(lay, n, i, 1e-2).numpy() for i in range(K)])
+    compare_states(dev, ref, "side stream")
+    assert_same(w_out, ref.w, "w read back by the last step, which was a host step")
