@@ -243,6 +243,19 @@ ssd_status ssd_advance(ssd_ctx *ctx);
  * that push and local update only read the gradient, Section 2.2). */
 ssd_status ssd_step(ssd_ctx *ctx, const void *const *grads, void *cuda_stream);
 
+/* ssd_step restricted to the tensors [first_tensor, first_tensor + num_tensors) of the
+ * layout (their arena range, padding included), at the context's current
+ * iteration, WITHOUT moving the counters.  The paper's training pipeline pushes and
+ * updates layer by layer while the backward pass is still producing the gradients
+ * of earlier layers (Section 2.1); this is the call for that: enqueue one group of
+ * layers as soon as their gradients are ready, in any order, each tensor exactly
+ * once per iteration, then call ssd_advance.  The update is elementwise, so the
+ * result equals one ssd_step over the whole arena, bit for bit.  `grads` are the K
+ * whole gradient arenas, as for ssd_step.  One kernel launch per call (none when
+ * the tensors are all empty).  Errors: SSD_ERR_ARG (range outside the layout). */
+ssd_status ssd_step_tensors(ssd_ctx *ctx, const void *const *grads, int32_t first_tensor,
+                            int32_t num_tensors, void *cuda_stream);
+
 /* ssd_step for gradients that arrive in HOST memory (as they would from a
  * network push).  `host_grads`: K host pointers (pinned memory, or the copies are
  * not asynchronous); `staging`: K device buffers of arena size (gradient dtype) that

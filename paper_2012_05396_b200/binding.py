@@ -31,7 +31,7 @@ SSD_MAX_WORKERS = 32
 EXPORTS = (
     "ssd_arena_numel", "ssd_init", "ssd_destroy", "ssd_tensor_offset", "ssd_schedule",
     "ssd_server_sync_update", "ssd_server_sync_update_static", "ssd_worker_glu_update", "ssd_worker_local_step", "ssd_advance",
-    "ssd_step", "ssd_step_host", "ssd_broadcast_weights", "ssd_worker_weights", "ssd_get_counters",
+    "ssd_step", "ssd_step_tensors", "ssd_step_host", "ssd_broadcast_weights", "ssd_worker_weights", "ssd_get_counters",
     "ssd_set_counters", "ssd_set_lr", "ssd_tensor_table_bytes", "ssd_set_tensor_scales", "ssd_get_hparams", "ssd_set_launch", "ssd_set_kernel_shape",
     "ssd_kernel_launches",
     "ssd_status_str", "ssd_last_cuda_error",
@@ -86,6 +86,7 @@ def lib():
             "ssd_worker_local_step": (i32, [vp, i32, vp, vp]),
             "ssd_advance": (i32, [vp]),
             "ssd_step": (i32, [vp, P(vp), vp]),
+            "ssd_step_tensors": (i32, [vp, P(vp), i32, i32, vp]),
             "ssd_step_host": (i32, [vp, P(vp), P(vp), vp, vp]),
             "ssd_broadcast_weights": (i32, [vp, vp]),
             "ssd_worker_weights": (i32, [vp, i32, P(vp), P(i32)]),
@@ -227,6 +228,10 @@ class Context:
 
     def ssd_step(self, grads: Sequence, stream=None):
         self._check(lib().ssd_step(self._h, _ptr_table(grads), _stream(stream)), "ssd_step")
+
+    def ssd_step_tensors(self, grads: Sequence, first_tensor: int, num_tensors: int, stream=None):
+        self._check(lib().ssd_step_tensors(self._h, _ptr_table(grads), first_tensor, num_tensors,
+                                           _stream(stream)), "ssd_step_tensors")
 
     def ssd_step_host(self, host_grads: Sequence, staging: Sequence, host_w_out=None, stream=None):
         self._check(lib().ssd_step_host(self._h, _ptr_table(host_grads), _ptr_table(staging),

@@ -214,7 +214,7 @@ Shape sync_shape(const ssd_ctx *c, bool wide_ok)
     return finish_shape(c, sh, wide_ok, 8);
 }
 
-Shape step_shape(const ssd_ctx *c, int flags, bool wide_ok)
+Shape step_shape(const ssd_ctx *c, int flags, bool wide_ok, int64_t count)
 {
     // Iterations that add K stores per element (pull; refresh or first call with one pre_weight
     // per worker) are write-heavy: 512 threads per SM.  The others: 640 threads per SM.
@@ -225,7 +225,7 @@ Shape step_shape(const ssd_ctx *c, int flags, bool wide_ok)
     // DRAM: smaller vectors spread it over more threads, and two workers' loads per thread halve the
     // number of dependent round trips.
     const int64_t sg = c->hp.grad_dtype == SSD_BF16 ? 2 : 4;
-    if (c->n * (c->hp.K * (sg + 12) + 16) < kL2ResidentBytes) sh = Shape{4, 2, 64, 0};
+    if (count * (c->hp.K * (sg + 12) + 16) < kL2ResidentBytes) sh = Shape{4, 2, 64, 0};
     return finish_shape(c, sh, wide_ok, 4);
 }
 
@@ -326,7 +326,8 @@ ssd_status launch_sync(ssd_ctx *c, const void *const *grads, int flags, cudaStre
     const bool state32 = (flags & kCopy) ? c->state32 : (aligned32(c->w) && aligned32(c->mom));
     p.tt = table_of(c);
     p.tt.base = lo;
-    const Shape sh = sync_shape(c, can_use_256bit(c, state32, grads, c->hp.K));
+    // a range that starts 4 elements off an 8-element boundary is only 16-byte aligned
+    const Shape sh = sync_shape(c, lo % 8 == 0 && can_use_256bit(c, state32, grads, c->hp.K));
     return p.tt.T ? launch_sync_t<true>(c, p, sh, stream) : launch_sync_t<false>(c, p, sh, stream);
 }
 
@@ -395,7 +396,7 @@ ssd_status launch_step(ssd_ctx *c, const void *const *grads, int flags, cudaStre
     p.s = c->s;
     p.tt = table_of(c);
     p.tt.base = lo;
-    const Shape sh = step_shape(c, flags, can_use_256bit(c, c->state32, grads, c->hp.K));
+    const Shape sh = step_shape(c, flags, lo % 8 == 0 && can_use_256bit(c, c->state32, grads, c->hp.K), p.n);
     return p.tt.T ? launch_step_t<true>(c, p, sh, stream) : launch_step_t<false>(c, p, sh, stream);
 }
 
@@ -677,6 +678,24 @@ ssd_status ssd_step(ssd_ctx *ctx, const void *const *grads, void *cuda_stream)
     if (st != SSD_OK) return st;
     advance(ctx);
     return SSD_OK;
+}
+
+ssd_status ssd_step_tensors(ssd_ctx *ctx, const void *const *grads, int32_t first_tensor, int32_t num_tensors,
+                            void *cuda_stream)
+{
+    if (!ctx) return SSD_ERR_ARG;
+    ssd_status st = check_grads(ctx, grads);
+    if (st != SSD_OK) return st;
+    const int32_t T = static_cast<int32_t>(ctx->offsets.size());
+    if (first_tensor < 0 || num_tensors < 1 || first_tensor > T - num_tensors) return SSD_ERR_ARG;
+    const int64_t lo = ctx->offsets[first_tensor];
+    const int64_t hi = first_tensor + num_tensors < T ? ctx->offsets[first_tensor + num_tensors] : ctx->n;
+    if (hi == lo) return SSD_OK;                      // only empty tensors
+    int32_t stage, flags;
+    schedule_of(ctx, ctx->iter, &stage, &flags);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    return (stage == SSD_STAGE_WARMUP) ? launch_sync(ctx, grads, flags & SSD_FLAG_COPY, stream, lo, hi - lo)
+                                       : launch_step(ctx, grads, flags, stream, lo, hi - lo);
 }
 
 ssd_status ssd_step_host(ssd_ctx *ctx, const void *const *host_grads, void *const *staging,

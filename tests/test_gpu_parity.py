@@ -463,3 +463,50 @@ def test_work_is_ordered_on_the_callers_stream():
         ref.step([synth.gradient(lay, n, i, 1e-2).numpy() for i in range(K)])
     compare_states(dev, ref, "side stream")
     assert_same(w_out, ref.w, "w read back by the last step, which was a host step")
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_layer_by_layer_stepping_equals_one_step(bf16):
+    # groups of tensors updated in reverse network order (the order in which a backward pass delivers
+    # gradients), with group boundaries that are only 16-byte aligned, per-tensor scales and a shared
+    # pre_weight; every iteration must equal one ssd_step over the whole arena
+    K, W, k, iters = 3, 2, 2, 8
+    lay = synth.Layout("t")
+    for i, cnt in enumerate((5, 1, 10, 3, 64, 7, 1024, 2, 36, 4100, 12, 9, 20000, 4, 4, 33)):
+        lay.add(f"x{i}", cnt, "he" if i % 3 else "zero", 16)
+    T = lay.num_tensors
+    _, chp = make_hp(K, 0.1, 0.9, W, k, wd=1e-3, bf16=bf16)
+    w0 = synth.init_weights(lay)
+    whole = DeviceState(lay.numels, chp, w0, shared_pre=True)
+    layered = DeviceState(lay.numels, chp, w0, shared_pre=True)
+    wd_mult = [1.0 if kind == "he" else 0.0 for kind in lay.kinds]
+    tables = [torch.empty(s.ctx.ssd_tensor_table_bytes(), dtype=torch.uint8, device="cuda") for s in (whole, layered)]
+    whole.ctx.ssd_set_tensor_scales(None, wd_mult, tables[0])
+    layered.ctx.ssd_set_tensor_scales(None, wd_mult, tables[1])
+    assert any(o % 8 == 4 for o in lay.offsets)            # some groups start off the 256-bit grid
+    groups, t = [], 0
+    for size in itertools.cycle((1, 3, 2, 7)):
+        if t >= T:
+            break
+        groups.append((t, min(size, T - t)))
+        t += size
+    for n in range(iters):
+        grads = [synth.gradient(lay, n, i, 1e-2, device="cuda") for i in range(K)]
+        if bf16:
+            grads = [synth.to_bf16(g) for g in grads]
+        whole.ctx.ssd_step(grads)
+        for first, count in reversed(groups):
+            layered.ctx.ssd_step_tensors(grads, first, count)
+        layered.ctx.ssd_advance()
+        torch.cuda.synchronize()
+        for name in ("w", "mom"):
+            assert torch.equal(getattr(whole, name).view(torch.int32), getattr(layered, name).view(torch.int32)), (name, n)
+        for i in range(K):
+            for name in ("w_loc", "pre", "w_dev"):
+                assert torch.equal(getattr(whole, name)[i].view(torch.int32),
+                                   getattr(layered, name)[i].view(torch.int32)), (name, i, n)
+    assert whole.ctx.ssd_get_counters() == layered.ctx.ssd_get_counters()
+    assert layered.ctx.ssd_kernel_launches() == iters * len(groups)
+    with pytest.raises(B.SsdError) as e:
+        layered.ctx.ssd_step_tensors(grads, T - 1, 2)
+    assert e.value.status == B.SSD_ERR_ARG
