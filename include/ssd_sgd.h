@@ -33,6 +33,9 @@
  *    runtime itself (ssd_last_cuda_error has its text); no counter moved, but
  *    work enqueued before the failing call stays enqueued.
  *  - A context is not thread-safe; use one per host thread or lock around it.
+ *    It works on the CUDA device that is current when its first launching call is
+ *    made (the device its buffers live on); keep that device current for every
+ *    later call on the context.
  *
  * Arena layout.  A parameter layout is an ordered list of T tensors given by
  * their element counts.  Tensor t lives at element offset ssd_tensor_offset(t)
