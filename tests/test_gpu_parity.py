@@ -510,3 +510,53 @@ def test_layer_by_layer_stepping_equals_one_step(bf16):
     with pytest.raises(B.SsdError) as e:
         layered.ctx.ssd_step_tensors(grads, T - 1, 2)
     assert e.value.status == B.SSD_ERR_ARG
+
+
+def test_random_combinations_of_every_option():
+    # seeded draw over layouts, K, schedule, gradient type, per-tensor scales, shared pre_weight, local
+    # updater, kernel shape and the way an iteration is issued (whole step, layer groups, split calls)
+    rng = np.random.default_rng(20201205)
+    for case in range(40):
+        T = int(rng.integers(1, 9))
+        numels = [int(rng.choice([0, 1, 3, 4, 5, 8, 17, 64, 100, 1000, 4099])) for _ in range(T)]
+        if sum(numels) == 0:
+            numels[0] = 6
+        K = int(rng.choice([1, 2, 3, 4, 7, 8, 16, 32]))
+        W, k = int(rng.integers(0, 4)), int(rng.integers(0, 5))
+        bf16, per_tensor = bool(rng.integers(2)), bool(rng.integers(2))
+        local_sgd = bool(rng.integers(4) == 0)
+        shared = bool(rng.integers(2)) and K > 1 and k > 0
+        issue = str(rng.choice(["step", "layers"] if shared else ["step", "layers", "split"]))
+        vw, batch = int(rng.choice([0, 4, 8])), int(rng.choice([0, 1, 2, 4, 8]))
+        iters = W + 2 * max(k, 1) + 2
+        tag = f"case {case}: numels={numels} K={K} W={W} k={k} bf16={bf16} pt={per_tensor} sgd={local_sgd} " \
+              f"shared={shared} issue={issue} shape=({vw},{batch})"
+        lay = synth.Layout("t")
+        for i, cnt in enumerate(numels):
+            lay.add(f"x{i}", cnt, "he", 8)
+        ohp, chp = make_hp(K, 0.1, 0.9, W, k, wd=0.01, bf16=bf16, local_sgd=local_sgd)
+        w0 = synth.init_weights(lay, seed=case)
+        dev = DeviceState(lay.numels, chp, w0, shared_pre=shared)
+        dev.ctx.ssd_set_kernel_shape(vw, batch)
+        if per_tensor:
+            lr_mult = [float(x) for x in rng.choice([0.25, 0.5, 1.0, 2.0], T)]
+            wd_mult = [float(x) for x in rng.choice([0.0, 1.0, 3.0], T)]
+            ohp.set_tensor_scales(tensor_ends(lay), lr_mult, wd_mult)
+            table = torch.empty(dev.ctx.ssd_tensor_table_bytes(), dtype=torch.uint8, device="cuda")
+            dev.ctx.ssd_set_tensor_scales(lr_mult, wd_mult, table)
+        ref = oracle.State(ohp, w0.numpy())
+        for n in range(iters):
+            grads = [synth.gradient(lay, n, i, 0.05, seed=case, device="cuda") for i in range(K)]
+            if bf16:
+                grads = [synth.to_bf16(g) for g in grads]
+            if issue == "step":
+                dev.ctx.ssd_step(grads)
+            elif issue == "layers":
+                for t in reversed(range(T)):
+                    dev.ctx.ssd_step_tensors(grads, t, 1)
+                dev.ctx.ssd_advance()
+            else:
+                gpu_iteration(dev, grads, "split")
+            ref.step([oracle_grad(g, bf16) for g in grads])
+        torch.cuda.synchronize()
+        compare_states(dev, ref, tag)
