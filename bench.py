@@ -52,7 +52,7 @@ NCU_TRAFFIC = {"digest": "e88e800962cb2a50", "workload": "vgg16_K16",
 
 def kernel_digest() -> str:
     h = hashlib.sha256()
-    for name in ("ssd_kernels.cuh", "ssd_sgd.cu"):
+    for name in ("ssd_kernels.cuh", "ssd_ring.cuh", "ssd_sgd.cu"):
         with open(os.path.join(ROOT, "paper_2012_05396_b200", "csrc", name), "rb") as fh:
             h.update(fh.read())
     return h.hexdigest()[:16]

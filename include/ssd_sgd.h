@@ -333,6 +333,20 @@ ssd_status ssd_set_launch(ssd_ctx *ctx, int32_t threads_per_block, int32_t block
  * the alignment and K.  Results do not depend on either. */
 ssd_status ssd_set_kernel_shape(ssd_ctx *ctx, int32_t vector_elems, int32_t batch);
 
+/* Shared-memory staging for the fused step.  stages = 2..8 makes ssd_step (and its
+ * range forms) in the delay stage use a kernel in which one thread per block streams
+ * the inputs into a ring of `stages` shared-memory buffers with bulk asynchronous
+ * copies and 256 threads consume them; 0 (the default) is the register path.  On
+ * B200 the register path is the faster one; the staged kernel is kept for comparison
+ * and gives the same bits.  Contexts with a shared pre_weight or the plain-SGD
+ * updater, and bfloat16 ranges that do not start and end on multiples of 8 elements,
+ * stay on the register path.  Every wait inside the staged kernel is bounded; if one
+ * ever runs out, the launch ends early with its results incomplete and
+ * ssd_staging_error reports 1 (process-wide, sticky; the call synchronises the
+ * device). */
+ssd_status ssd_set_staging(ssd_ctx *ctx, int32_t stages);
+ssd_status ssd_staging_error(ssd_ctx *ctx, int32_t *flag);
+
 /* Number of kernels this context has launched so far. */
 int64_t ssd_kernel_launches(const ssd_ctx *ctx);
 

@@ -33,7 +33,7 @@ EXPORTS = (
     "ssd_server_sync_update", "ssd_server_sync_update_static", "ssd_worker_glu_update", "ssd_worker_local_step", "ssd_advance",
     "ssd_step", "ssd_step_tensors", "ssd_step_host", "ssd_broadcast_weights", "ssd_worker_weights", "ssd_get_counters",
     "ssd_set_counters", "ssd_set_lr", "ssd_tensor_table_bytes", "ssd_set_tensor_scales", "ssd_get_hparams", "ssd_set_launch", "ssd_set_kernel_shape",
-    "ssd_kernel_launches",
+    "ssd_set_staging", "ssd_staging_error", "ssd_kernel_launches",
     "ssd_status_str", "ssd_last_cuda_error",
 )
 
@@ -98,6 +98,8 @@ def lib():
             "ssd_get_hparams": (i32, [vp, P(ssd_hparams), P(C.c_float)]),
             "ssd_set_launch": (i32, [vp, i32, i32]),
             "ssd_set_kernel_shape": (i32, [vp, i32, i32]),
+            "ssd_set_staging": (i32, [vp, i32]),
+            "ssd_staging_error": (i32, [vp, P(i32)]),
             "ssd_kernel_launches": (i64, [vp]),
             "ssd_status_str": (C.c_char_p, [i32]),
             "ssd_last_cuda_error": (C.c_char_p, [vp]),
@@ -282,6 +284,14 @@ class Context:
 
     def ssd_set_kernel_shape(self, vector_elems: int = 0, batch: int = 0):
         self._check(lib().ssd_set_kernel_shape(self._h, vector_elems, batch), "ssd_set_kernel_shape")
+
+    def ssd_set_staging(self, stages: int = 0):
+        self._check(lib().ssd_set_staging(self._h, stages), "ssd_set_staging")
+
+    def ssd_staging_error(self) -> int:
+        out = C.c_int32()
+        self._check(lib().ssd_staging_error(self._h, C.byref(out)), "ssd_staging_error")
+        return out.value
 
     def ssd_kernel_launches(self) -> int:
         return lib().ssd_kernel_launches(self._h)

@@ -10,7 +10,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libssd_sgd.so")
 SOURCES = [os.path.join(CSRC, "ssd_sgd.cu")]
-DEPENDS = SOURCES + [os.path.join(CSRC, "ssd_kernels.cuh"), os.path.join(ROOT, "include", "ssd_sgd.h")]
+DEPENDS = SOURCES + [os.path.join(CSRC, "ssd_kernels.cuh"), os.path.join(CSRC, "ssd_ring.cuh"), os.path.join(ROOT, "include", "ssd_sgd.h")]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",

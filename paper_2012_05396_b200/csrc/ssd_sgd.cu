@@ -3,6 +3,7 @@
 // The contract of every entry point is stated in include/ssd_sgd.h.
 #include "ssd_sgd.h"
 #include "ssd_kernels.cuh"
+#include "ssd_ring.cuh"
 
 #include <cmath>
 #include <cstring>
@@ -42,6 +43,7 @@ struct ssd_ctx {
     bool state32 = false;             // every state buffer is 32-byte aligned
     int threads = 0, blocks_per_sm = 0;     // 0: the kernel's default shape
     int force_vw = 0, force_batch = 0;      // 0: chosen from alignment and K
+    int staging = 0;                        // > 0: fused step through a shared-memory ring of that many stages
     // per-tensor scalars: host copies of the multipliers and the caller's device table
     std::vector<float> lr_mult, wd_mult;
     void *tensor_table = nullptr;
@@ -377,6 +379,44 @@ ssd_status launch_step_t(ssd_ctx *c, const StepParams &p, const Shape &sh, cudaS
     return bf16 ? launch_step_b<kBF16, 4, PT>(c, p, sh, stream) : launch_step_b<kF32, 4, PT>(c, p, sh, stream);
 }
 
+// The shared-memory ring covers the common case; the rest stays on the register path.  Its bulk
+// copies need 16-byte aligned sources and sizes, which bfloat16 gradients give only for ranges that
+// start and end on multiples of 8 elements.
+bool ring_can_run(const ssd_ctx *c, int64_t lo, int64_t count)
+{
+    if (c->shared_pre || c->hp.local_updater != SSD_LOCAL_GLU) return false;
+    if (c->hp.grad_dtype == SSD_BF16 && (lo % 8 != 0 || count % 8 != 0)) return false;
+    return true;
+}
+
+template <typename Kernel>
+ssd_status launch_ring(ssd_ctx *c, Kernel kernel, const StepParams &p, cudaStream_t stream)
+{
+    ssd_status st = ensure_device(c);
+    if (st != SSD_OK) return st;
+    const int stages = c->staging;
+    const size_t smem = static_cast<size_t>(stages) * kRingStageBytes + 2 * stages * sizeof(uint64_t);
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    const int64_t ntiles = (p.n + kRingTile - 1) / kRingTile;
+    const int grid = static_cast<int>(ntiles < c->dev.sms ? ntiles : c->dev.sms);    // one block per SM
+    kernel<<<grid, kRingThreads, smem, stream>>>(p, stages);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    c->launches += 1;
+    return SSD_OK;
+}
+
+ssd_status launch_step_ring(ssd_ctx *c, const StepParams &p, cudaStream_t stream)
+{
+    const bool bf16 = c->hp.grad_dtype == SSD_BF16;
+    if (p.tt.T)
+        return bf16 ? launch_ring(c, step_ring_kernel<kBF16, true>, p, stream)
+                    : launch_ring(c, step_ring_kernel<kF32, true>, p, stream);
+    return bf16 ? launch_ring(c, step_ring_kernel<kBF16, false>, p, stream)
+                : launch_ring(c, step_ring_kernel<kF32, false>, p, stream);
+}
+
 ssd_status launch_step(ssd_ctx *c, const void *const *grads, int flags, cudaStream_t stream,
                        int64_t lo = 0, int64_t count = -1)
 {
@@ -396,6 +436,7 @@ ssd_status launch_step(ssd_ctx *c, const void *const *grads, int flags, cudaStre
     p.s = c->s;
     p.tt = table_of(c);
     p.tt.base = lo;
+    if (c->staging && ring_can_run(c, lo, p.n)) return launch_step_ring(c, p, stream);
     const Shape sh = step_shape(c, flags, lo % 8 == 0 && can_use_256bit(c, c->state32, grads, c->hp.K), p.n);
     return p.tt.T ? launch_step_t<true>(c, p, sh, stream) : launch_step_t<false>(c, p, sh, stream);
 }
@@ -899,6 +940,24 @@ ssd_status ssd_set_kernel_shape(ssd_ctx *ctx, int32_t vector_elems, int32_t batc
     if (batch != 0 && batch != 1 && batch != 2 && batch != 4 && batch != 8) return SSD_ERR_ARG;
     ctx->force_vw = vector_elems;
     ctx->force_batch = batch;
+    return SSD_OK;
+}
+
+ssd_status ssd_set_staging(ssd_ctx *ctx, int32_t stages)
+{
+    if (!ctx) return SSD_ERR_ARG;
+    if (stages != 0 && (stages < 2 || stages > kRingMaxStages)) return SSD_ERR_ARG;
+    ctx->staging = stages;
+    return SSD_OK;
+}
+
+ssd_status ssd_staging_error(ssd_ctx *ctx, int32_t *flag)
+{
+    if (!ctx || !flag) return SSD_ERR_ARG;
+    int value = 0;
+    cudaError_t e = cudaMemcpyFromSymbol(&value, g_ring_error, sizeof value);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    *flag = value;
     return SSD_OK;
 }
 

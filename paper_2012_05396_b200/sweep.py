@@ -64,7 +64,7 @@ def _fits(nbytes):
 
 
 def point(log2n: int, K: int, dtype: str, kernels, reps: int, peak: float, threads: int, bps: int,
-          vw: int = 0, batch: int = 0):
+          vw: int = 0, batch: int = 0, staging: int = 0):
     n = 1 << log2n
     sg = 2 if dtype == "bf16" else 4
     out = []
@@ -86,6 +86,8 @@ def point(log2n: int, K: int, dtype: str, kernels, reps: int, peak: float, threa
             st.ctx.ssd_set_launch(threads, bps)
         if vw or batch:
             st.ctx.ssd_set_kernel_shape(vw, batch)
+        if staging:
+            st.ctx.ssd_set_staging(staging)       # fused step through the shared-memory ring
 
     w0 = synth.uniform_buffer(synth.STREAM_WEIGHT, n, device="cuda")
     if "sync" in kernels:
@@ -164,6 +166,8 @@ def main():
     ap.add_argument("--blocks-per-sm", type=int, default=0)
     ap.add_argument("--vector-elems", type=int, default=0, choices=[0, 4, 8])
     ap.add_argument("--batch", type=int, default=0, choices=[0, 1, 2, 4, 8])
+    ap.add_argument("--staging", type=int, default=0,
+                    help="stages of the shared-memory ring for the fused step (0 = register path)")
     args = ap.parse_args()
     if not torch.cuda.is_available():
         raise SystemExit("the sweep needs a CUDA device")
@@ -172,7 +176,7 @@ def main():
         for K in args.K:
             for dtype in args.dtype:
                 for rec in point(log2n, K, dtype, args.kernels, args.reps, args.peak, args.threads,
-                                 args.blocks_per_sm, args.vector_elems, args.batch):
+                                 args.blocks_per_sm, args.vector_elems, args.batch, args.staging):
                     print(json.dumps(rec), flush=True)
 
 

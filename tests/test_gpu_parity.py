@@ -560,3 +560,46 @@ def test_random_combinations_of_every_option():
             ref.step([oracle_grad(g, bf16) for g in grads])
         torch.cuda.synchronize()
         compare_states(dev, ref, tag)
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_staged_step_kernel_gives_the_same_bits(bf16):
+    # the bulk-copy / shared-memory ring variant of the fused step: every flag of the schedule, several
+    # ring depths, per-tensor scalars, tiles with a ragged end, layer-group ranges
+    K, W, k, iters = 4, 1, 3, 9
+    lay = synth.Layout("t")
+    for i, cnt in enumerate((5000, 3, 2048, 64, 4100, 12, 8)):
+        lay.add(f"x{i}", cnt, "he", 16)
+    ohp, chp = make_hp(K, 0.1, 0.9, W, k, wd=0.01, bf16=bf16)
+    lr_mult = [1.0, 0.5, 2.0, 1.0, 0.25, 1.0, 4.0]
+    wd_mult = [1.0, 0.0, 3.0, 0.0, 1.0, 0.0, 2.0]
+    w0 = synth.init_weights(lay)
+    for stages, per_tensor, layers in ((2, False, False), (3, True, False), (8, False, True), (4, True, True)):
+        if per_tensor:
+            ohp.set_tensor_scales(tensor_ends(lay), lr_mult, wd_mult)
+        else:
+            ohp.tensor_end = None
+        dev = DeviceState(lay.numels, chp, w0)
+        dev.ctx.ssd_set_staging(stages)
+        if per_tensor:
+            table = torch.empty(dev.ctx.ssd_tensor_table_bytes(), dtype=torch.uint8, device="cuda")
+            dev.ctx.ssd_set_tensor_scales(lr_mult, wd_mult, table)
+        ref = oracle.State(ohp, w0.numpy())
+        for n in range(iters):
+            grads = [synth.gradient(lay, n, i, 0.05, device="cuda") for i in range(K)]
+            if bf16:
+                grads = [synth.to_bf16(g) for g in grads]
+            if layers:
+                for first, count in ((4, 3), (1, 3), (0, 1)):
+                    dev.ctx.ssd_step_tensors(grads, first, count)
+                dev.ctx.ssd_advance()
+            else:
+                dev.ctx.ssd_step(grads)
+            ref.step([oracle_grad(g, bf16) for g in grads])
+            torch.cuda.synchronize()
+            compare_states(dev, ref, f"ring stages={stages} pt={per_tensor} layers={layers} iter {n}")
+        assert dev.ctx.ssd_staging_error() == 0
+    with pytest.raises(B.SsdError):
+        dev.ctx.ssd_set_staging(9)
+    with pytest.raises(B.SsdError):
+        dev.ctx.ssd_set_staging(1)
