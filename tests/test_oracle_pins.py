@@ -592,3 +592,27 @@ def test_local_sgd_equals_glu_with_alpha_one_beta_zero():
     for i in range(K):
         np.testing.assert_array_equal(a.w_loc[i], b.w_loc[i])
         np.testing.assert_array_equal(a.w_dev[i], b.w_dev[i])
+
+
+def test_brute_force_random_hyper_parameters():
+    # the scalar rewrite against the oracle on random hyper-parameters, not only the paper's defaults
+    rng = np.random.default_rng(16)
+    for _ in range(25):
+        K, N, T = int(rng.integers(1, 6)), int(rng.integers(1, 9)), 9
+        W, k = int(rng.integers(0, 4)), int(rng.integers(0, 5))
+        lr, m = float(rng.uniform(0.01, 0.5)), float(rng.uniform(0.0, 0.95))
+        wd, lr_loc = float(rng.uniform(0.0, 0.1)), float(rng.uniform(0.01, 1.0))
+        alpha, beta = float(rng.uniform(0.0, 3.0)), float(rng.uniform(0.0, 2.0))
+        w0 = rng.standard_normal(N).astype(f32)
+        stream = [rng_grads(rng, K, N, 0.1) for _ in range(T)]
+        hp = Hyper(K=K, lr=lr, m=m, W=W, k=k, wd=wd, lr_loc=lr_loc, alpha=alpha, beta=beta)
+        st, _ = run_config(hp, w0, stream)
+        w, mom, w_loc, pre, w_dev = brute_force(K, lr, m, wd, W, k, lr_loc, alpha, beta, w0, stream)
+        np.testing.assert_array_equal(st.w, np.array(w, f32))
+        np.testing.assert_array_equal(st.mom, np.array(mom, f32))
+        for i in range(K):
+            np.testing.assert_array_equal(st.w_loc[i], np.array(w_loc[i], f32))
+            if pre[i][0] is not None:
+                np.testing.assert_array_equal(st.pre[i], np.array(pre[i], f32))
+            if w_dev[i][0] is not None:
+                np.testing.assert_array_equal(st.w_dev[i], np.array(w_dev[i], f32))
