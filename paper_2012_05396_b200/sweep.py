@@ -23,7 +23,7 @@ import torch
 from . import binding as B
 from . import build as libbuild
 from . import synth
-from .state import DeviceState
+from .state import DeviceState, alloc_arenas
 
 L2_BYTES = 126e6
 
@@ -44,11 +44,11 @@ def time_launches(fn, reps: int, warmup: int = 3):
 
 
 def _grads(n, K, dtype):
-    out = []
+    out = alloc_arenas(K, n, torch.bfloat16 if dtype == "bf16" else torch.float32)
     for i in range(K):
         g = synth.uniform_buffer(synth.STREAM_GRAD, n, worker=i, device="cuda")
         g.mul_(1e-3)                     # keeps the state bounded over many repetitions
-        out.append(synth.to_bf16(g) if dtype == "bf16" else g)
+        out[i].copy_(g)                  # rounds to nearest even for bfloat16
     return out
 
 
