@@ -8,8 +8,10 @@ launches, median and minimum reported):
     glu     ssd_worker_glu_update, plain flags   sg + 12 bytes per parameter and worker
     step    ssd_step in the steps-delay stage    K*(sg+12) + 16 (+4K on refresh, +4K on pull)
 and prints one JSON object per point.  State and gradients are uniform(-1,1) from the seeded
-generators.  Points whose footprint is below four times the L2 size are marked "l2": they are not
-HBM measurements.  Points that do not fit in free device memory are reported as skipped.
+generators.  Points whose footprint is below 1 GB rotate over several independent buffer sets (at
+least 1 GB together), so that a launch never finds its data in the 126 MB L2 left by the previous
+one; points below four times the L2 size are still marked "l2" (they last microseconds and show
+launch latency).  Points that do not fit in free device memory are reported as skipped.
 """
 from __future__ import annotations
 
@@ -59,6 +61,7 @@ def _hp(K, k, dtype):
 
 
 def _fits(nbytes):
+    torch.cuda.empty_cache()             # blocks cached from the previous point count as free
     free, _ = torch.cuda.mem_get_info()
     return nbytes * 1.03 + (1 << 30) <= free
 
@@ -89,23 +92,38 @@ def point(log2n: int, K: int, dtype: str, kernels, reps: int, peak: float, threa
         if staging:
             st.ctx.ssd_set_staging(staging)       # fused step through the shared-memory ring
 
+    def copies(footprint):
+        """Independent buffer sets to rotate over, so that no launch finds its data in the 126 MB L2:
+        at least 1 GB in total (at most 8 sets)."""
+        return max(1, min(8, -(-int(1e9) // footprint)))
+
     w0 = synth.uniform_buffer(synth.STREAM_WEIGHT, n, device="cuda")
     if "sync" in kernels:
         # the server alone: a context without a delay stage needs no worker state
         fp = 2 * n * 4 + K * n * sg
-        if _fits(fp):
-            st = DeviceState([n], _hp(K, 0, dtype), w0, worker_state=False)
-            tune(st)
-            grads = _grads(n, K, dtype)
-            med, mn = time_launches(lambda: st.ctx.ssd_server_sync_update(grads), reps)
+        R = copies(fp)
+        if _fits(fp * R):
+            sets = []
+            for _ in range(R):
+                st = DeviceState([n], _hp(K, 0, dtype), w0, worker_state=False)
+                tune(st)
+                sets.append((st, _grads(n, K, dtype)))
+            turn = {"i": 0}
+
+            def sync():
+                st, grads = sets[turn["i"]]
+                st.ctx.ssd_server_sync_update(grads)
+                turn["i"] = (turn["i"] + 1) % R
+            med, mn = time_launches(sync, reps)
             emit("sync", fp, (K * sg + 16) * n, med, mn)
-            del st, grads
+            del sets
         else:
             skip("sync", fp)
     if "glu" in kernels:
-        # one launch updates one worker, so the worker count does not enter; rotate over up to
-        # four workers' buffers so that consecutive launches touch different memory
-        Kg = min(K, 4)
+        # one launch updates one worker, so the worker count does not enter; rotate over the buffers
+        # of enough workers that consecutive launches never touch the same memory
+        fp1 = 3 * n * 4 + n * sg                     # one worker's buffers
+        Kg = max(min(K, 4), min(8, -(-int(1e9) // fp1)))
         fp = (2 + 3 * Kg) * n * 4 + Kg * n * sg
         if _fits(fp):
             st = DeviceState([n], _hp(Kg, 4, dtype), w0, fill=0.0)
@@ -126,28 +144,32 @@ def point(log2n: int, K: int, dtype: str, kernels, reps: int, peak: float, threa
             skip("glu", fp)
     if "step" in kernels:
         fp = (2 + 3 * K) * n * 4 + K * n * sg
-        if _fits(fp):
-            st = DeviceState([n], _hp(K, 4, dtype), w0, fill=0.0)
-            tune(st)
-            grads = _grads(n, K, dtype)
-            st.ctx.ssd_step(grads)                                   # first GLU call
+        R = copies(fp)
+        if _fits(fp * R):
+            sets = []
+            for _ in range(R):
+                st = DeviceState([n], _hp(K, 4, dtype), w0, fill=0.0)
+                tune(st)
+                grads = _grads(n, K, dtype)
+                st.ctx.ssd_step(grads)                               # first GLU call
+                sets.append((st, grads))
             stream = torch.cuda.current_stream()
             per_flag = {}
-            for _ in range(4):
-                st.ctx.ssd_step(grads)
-            for _ in range(max(reps, 8)):
+            for r in range(R * (4 + max(reps, 8))):                  # every set goes through the same schedule
+                st, grads = sets[r % R]
                 flags = st.ctx.ssd_get_counters()[3]
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record(stream)
                 st.ctx.ssd_step(grads)
                 e1.record(stream)
                 torch.cuda.synchronize()
-                per_flag.setdefault(flags, []).append(e0.elapsed_time(e1))
+                if r >= 4 * R:
+                    per_flag.setdefault(flags, []).append(e0.elapsed_time(e1))
             for flags, ms in sorted(per_flag.items()):
                 b = K * (sg + 12) + 16 + (4 * K if flags & 2 else 0) + (4 * K if flags & 4 else 0)
                 name = "step" + ("+refresh" if flags & 2 else "") + ("+pull" if flags & 4 else "")
                 emit(name, fp, b * n, statistics.median(ms), min(ms))
-            del st, grads
+            del sets
         else:
             skip("step", fp)
     torch.cuda.empty_cache()
