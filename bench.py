@@ -179,6 +179,32 @@ def oracle_sample_run(wl, n_sample: int, steps: int, grads_host, w0_host):
     return dt, moved, n_sample * steps, 1
 
 
+def oracle_all_cores_run(wl, n_sample: int, steps: int, grads_host, w0_host, threads: int):
+    """The same oracle, untouched, run by `threads` host threads on disjoint element ranges of the
+    sample (the update is elementwise; the C calls release the interpreter lock).  Returns seconds."""
+    import oracle
+    from concurrent.futures import ThreadPoolExecutor
+    hp = oracle.Hyper(K=wl["K"], lr=wl["lr"], m=wl["m"], W=wl["W"], k=wl["k"])
+    bounds = [n_sample * t // threads for t in range(threads + 1)]
+    parts = []
+    for t in range(threads):
+        lo, hi = bounds[t], bounds[t + 1]
+        st = oracle.State(hp, w0_host[lo:hi], fill=0.0)
+        gs = [[np.ascontiguousarray(g[lo:hi]) for g in gset] for gset in grads_host]
+        parts.append((st, gs))
+
+    def advance(part, first, count):
+        st, gs = part
+        for n in range(first, first + count):
+            st.step(gs[n % len(gs)])
+
+    with ThreadPoolExecutor(threads) as pool:
+        list(pool.map(lambda part: advance(part, 0, wl["W"] + 1), parts))       # untimed, as above
+        t0 = time.perf_counter()
+        list(pool.map(lambda part: advance(part, wl["W"] + 1, steps), parts))
+        return time.perf_counter() - t0
+
+
 def run_reference(args, wl_name, wl):
     """--impl reference: the CPU oracle on the host cores, a bounded sample per step."""
     from paper_2012_05396_b200 import synth
@@ -397,6 +423,11 @@ def main():
             "value": moved / dt / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
             "host_cores": os.cpu_count(), "params_per_s": params / dt, "ms_per_step_sample": dt / o_steps * 1e3,
             "sample": f"first {n_sample} of {N} arena elements, all {K} workers, {o_steps} delay-stage steps"}
+        threads = os.cpu_count() or 1
+        if threads > 1:
+            dt_all = oracle_all_cores_run(wl, n_sample, o_steps, g_host, w_host, threads)
+            line["cpu_baseline"]["all_cores"] = {"value": moved / dt_all / 1e9, "unit": UNIT, "cores": threads,
+                                                 "params_per_s": params / dt_all}
 
     if rank == 0:
         print(json.dumps(line))
