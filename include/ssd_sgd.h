@@ -27,8 +27,13 @@
  *    written below, the K gradients summed left to right (worker 0 first).
  *    Results are therefore unique and reproducible bit for bit.
  *  - Calls only enqueue work on `cuda_stream` (a cudaStream_t passed as void*,
- *    NULL = the legacy default stream) and return; they never synchronise.
+ *    NULL = the legacy default stream) and return without waiting for the GPU.
  *    Work of successive calls on the same stream is ordered by the stream.
+ *    Three calls copy a small table out of ordinary (pageable) host memory of
+ *    the context: ssd_set_tensor_scales, ssd_set_lr while per-tensor scales are
+ *    set, and ssd_server_sync_update_static.  The CUDA runtime stages such a
+ *    copy before the call returns, which can wait for earlier copies on that
+ *    stream; nothing else in the library blocks the host.
  *  - Every call returns an ssd_status.  Arguments are validated before any
  *    launch: on an argument, alignment, layout or state error nothing was
  *    enqueued and no counter moved.  SSD_ERR_CUDA reports a failure of the CUDA
@@ -120,9 +125,12 @@ typedef struct {
 } ssd_hparams;
 
 /* Caller-owned device state.  w_loc, pre, w_dev: host arrays of K device pointers.
- * The K*3+2 buffers must not overlap each other or any gradient buffer.  With
- * delay_k == 0 (synchronous SGD only) no worker state is ever touched and the
- * three tables may be NULL.
+ * The K*3+2 buffers must not overlap each other or any gradient buffer: ssd_init
+ * compares their byte ranges and every call that takes gradients compares those
+ * with the state (SSD_ERR_ARG).  With delay_k == 0 (synchronous SGD only) no
+ * worker state is ever touched and the three tables may be NULL.
+ * `pre` alone may be NULL when pre_weight is not to live in device memory: see
+ * ssd_set_host_pre_weight (or the plain-SGD local updater, which has none).
  * Shared pre_weight: the K pre_weight buffers always hold equal values (each worker
  * sets its own from the same pulled global weight: "the same pre_weight", Section
  * 3.3), so all K entries of `pre` may point at ONE buffer.  ssd_step then reads it
@@ -203,6 +211,7 @@ ssd_status ssd_server_sync_update(ssd_ctx *ctx, const void *const *grads, void *
  *    SSD_ERR_TOO_LARGE before anything is enqueued.
  *  - The first call on each device looks up the array's device address (with that
  *    device current).  Make that first call before starting any stream capture.
+ *    The context's device must be the current one (SSD_ERR_STATE otherwise).
  *  - The array is shared by every context and every call in the process and keeps
  *    what the last call wrote; each call overwrites the entries it uses.  Two calls
  *    whose work can overlap on the GPU (different streams, or different contexts on
@@ -266,14 +275,55 @@ ssd_status ssd_step_tensors(ssd_ctx *ctx, const void *const *grads, int32_t firs
  * not asynchronous); `staging`: K device buffers of arena size (gradient dtype) that
  * receive them; `host_w_out`: optional host buffer that receives the new global
  * weight w (NULL = no read-back).  The arena is processed in chunks of 2^24
- * elements: the host-to-device copies of one chunk, the update of the previous one
+ * elements (ssd_set_host_chunk): the host-to-device copies of one chunk, the update of the previous one
  * and the device-to-host copy of the one before overlap, on two side streams that
  * the context creates at the first call (driver objects, no device memory).  All of
  * it is ordered after the work already on `cuda_stream`, and `cuda_stream` ends
  * behind the last copy: the caller synchronises `cuda_stream` before reading
- * host_w_out or reusing host_grads.  One kernel launch per chunk. */
+ * host_w_out or reusing host_grads.  One kernel launch per chunk.  Errors:
+ * SSD_ERR_ARG, SSD_ERR_ALIGN, SSD_ERR_STATE (delay stage of a context without
+ * pre_weight buffers and without ssd_set_host_pre_weight), SSD_ERR_CUDA. */
 ssd_status ssd_step_host(ssd_ctx *ctx, const void *const *host_grads, void *const *staging,
                          float *host_w_out, void *cuda_stream);
+
+/* Elements per chunk of ssd_step_host: a multiple of 1024, at most 2^30; 0 = the
+ * default 2^24.  Results do not depend on it.  SSD_ERR_STATE while a host-resident
+ * pre_weight is set (its device slices were sized for the current chunk). */
+ssd_status ssd_set_host_chunk(ssd_ctx *ctx, int64_t chunk_elems);
+
+/* pre_weight in HOST memory.  The paper keeps the backup of the pulled weights
+ * (pre_weight) in CPU-side memory so that it does not occupy the accelerator
+ * (Section 3.5, "Embedding in Framework").  For a context created with
+ * ssd_buffers.pre == NULL this call names where it lives instead:
+ *   host_pre       ONE host arena of ssd_arena_numel() floats (pinned memory, or the
+ *                  copies are not asynchronous), 16-byte aligned.  One arena serves
+ *                  all K workers, whose pre_weights always hold equal values (see
+ *                  "Shared pre_weight" above).  The library reads and writes it;
+ *                  its content is part of the state (keep it across a checkpoint).
+ *   device_slices  device memory of slots * chunk floats (chunk = the ssd_step_host
+ *                  chunk, 2^24 unless changed), 16-byte aligned (32 for the 256-bit
+ *                  path), not overlapping any state buffer;
+ *   slots          1..8 slices; 2 or more let the copy of one chunk's slice overlap
+ *                  the update of the previous chunk.
+ * ssd_step_host then streams pre_weight with the gradients: per chunk, the slice is
+ * copied host-to-device next to the K gradient slices (except on the first GLU
+ * call, which does not read pre_weight), the fused step runs on the chunk with the
+ * slice as the one pre_weight of all workers, and on the iterations that overwrite
+ * pre_weight (first GLU call, refresh) the slice is copied back device-to-host on
+ * the side stream that also returns w.  Per step that is 4 bytes per parameter more
+ * host-to-device traffic (1/K of the gradients' when they are float32), 4 more
+ * device-to-host on one iteration in k, and K arenas of device memory less than
+ * private pre_weights (one less than a shared one).  Results equal the
+ * device-resident forms bit for bit.
+ * ssd_step_host also accepts host_grads == NULL in every mode: the gradients are
+ * then taken to be in `staging` already (device memory) and only pre_weight and w
+ * cross the bus.
+ * All other delay-stage calls (ssd_step, ssd_step_tensors, the per-worker calls)
+ * need pre_weight in device memory and return SSD_ERR_STATE for such a context.
+ * (NULL, NULL, 0) switches it off again.  Errors: SSD_ERR_ARG, SSD_ERR_ALIGN,
+ * SSD_ERR_STATE (the context has device pre_weight buffers, no worker state, or
+ * delay_k == 0). */
+ssd_status ssd_set_host_pre_weight(ssd_ctx *ctx, float *host_pre, float *device_slices, int32_t slots);
 
 /* w_loc[i] = w for every worker (the initial pull of Algorithm 1).  Needed before
  * the first step only when warmup_iters == 0.  One kernel launch.  SSD_ERR_STATE
@@ -323,17 +373,27 @@ ssd_status ssd_set_tensor_scales(ssd_ctx *ctx, const float *lr_mult, const float
 ssd_status ssd_get_hparams(const ssd_ctx *ctx, ssd_hparams *resolved, float *sync_scale);
 
 /* Launch shape of every kernel of this context: threads per block (multiple of
- * 32, 64..512) and resident blocks per SM (1..32, capped at what fits).  0 for
- * either returns it to the per-kernel default, which depends on the kernel, K,
- * the gradient type and the iteration's flags.  Results do not depend on it. */
+ * 32, 64..512) and resident blocks per SM (1..32, capped at what fits).  Each call
+ * sets both; 0 for either returns that one to the per-kernel default, which depends
+ * on the kernel, K, the gradient type and the iteration's flags.  Results do not
+ * depend on it. */
 ssd_status ssd_set_launch(ssd_ctx *ctx, int32_t threads_per_block, int32_t blocks_per_sm);
 
 /* Shape of the kernels' inner loop.  vector_elems: elements each thread owns per
- * trip, 8 (256-bit accesses; used only when every buffer involved is 32-byte
- * aligned, else 4 is taken) or 4 (128-bit); batch: workers whose loads a thread
- * issues together, 1, 2, 4 or 8 (the fused step uses at most 4).  0 = choose from
- * the alignment and K.  Results do not depend on either. */
+ * trip: 16 (two 256-bit accesses to float32 data, one to bfloat16 gradients), 8
+ * (one 256-bit access to float32 data, 128 bits of bfloat16) or 4 (128-bit); the
+ * wide forms are used only when every buffer involved is 32-byte aligned, else
+ * the next narrower one is taken.  batch: workers whose loads a thread issues
+ * together, 1, 2, 4 or 8 (the fused step uses at most 4, and at most 2 with
+ * vectors of 8 or 16, beyond which registers would spill; kernels with vectors of
+ * 16 run at most 256 threads per block).  0 = the default for the kernel, K,
+ * gradient type and alignment.  Results do not depend on either. */
 ssd_status ssd_set_kernel_shape(ssd_ctx *ctx, int32_t vector_elems, int32_t batch);
+
+/* The overrides as last set by ssd_set_launch and ssd_set_kernel_shape (0 = default).
+ * Outputs may be NULL. */
+ssd_status ssd_get_launch(const ssd_ctx *ctx, int32_t *threads_per_block, int32_t *blocks_per_sm,
+                          int32_t *vector_elems, int32_t *batch);
 
 /* Shared-memory staging for the fused step.  stages = 2..8 makes ssd_step (and its
  * range forms) in the delay stage use a kernel in which one thread per block streams

@@ -15,8 +15,7 @@ from typing import List, Optional, Sequence
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-# SSD_SGD_LIBRARY selects another build of the same library (e.g. one compiled with other cache hints)
-LIB_PATH = os.environ.get("SSD_SGD_LIBRARY") or os.path.join(_HERE, "libssd_sgd.so")
+LIB_PATH = os.path.join(_HERE, "libssd_sgd.so")
 
 (SSD_OK, SSD_ERR_ARG, SSD_ERR_ALIGN, SSD_ERR_LAYOUT, SSD_ERR_STATE, SSD_ERR_CUDA, SSD_ERR_NOMEM,
  SSD_ERR_TOO_LARGE) = range(8)
@@ -31,8 +30,8 @@ SSD_MAX_WORKERS = 32
 EXPORTS = (
     "ssd_arena_numel", "ssd_init", "ssd_destroy", "ssd_tensor_offset", "ssd_schedule",
     "ssd_server_sync_update", "ssd_server_sync_update_static", "ssd_worker_glu_update", "ssd_worker_local_step", "ssd_advance",
-    "ssd_step", "ssd_step_tensors", "ssd_step_host", "ssd_broadcast_weights", "ssd_worker_weights", "ssd_get_counters",
-    "ssd_set_counters", "ssd_set_lr", "ssd_tensor_table_bytes", "ssd_set_tensor_scales", "ssd_get_hparams", "ssd_set_launch", "ssd_set_kernel_shape",
+    "ssd_step", "ssd_step_tensors", "ssd_step_host", "ssd_set_host_chunk", "ssd_set_host_pre_weight", "ssd_broadcast_weights", "ssd_worker_weights", "ssd_get_counters",
+    "ssd_set_counters", "ssd_set_lr", "ssd_tensor_table_bytes", "ssd_set_tensor_scales", "ssd_get_hparams", "ssd_set_launch", "ssd_set_kernel_shape", "ssd_get_launch",
     "ssd_set_staging", "ssd_staging_error", "ssd_kernel_launches",
     "ssd_status_str", "ssd_last_cuda_error",
 )
@@ -88,6 +87,8 @@ def lib():
             "ssd_step": (i32, [vp, P(vp), vp]),
             "ssd_step_tensors": (i32, [vp, P(vp), i32, i32, vp]),
             "ssd_step_host": (i32, [vp, P(vp), P(vp), vp, vp]),
+            "ssd_set_host_chunk": (i32, [vp, i64]),
+            "ssd_set_host_pre_weight": (i32, [vp, vp, vp, i32]),
             "ssd_broadcast_weights": (i32, [vp, vp]),
             "ssd_worker_weights": (i32, [vp, i32, P(vp), P(i32)]),
             "ssd_get_counters": (i32, [vp, P(i64), P(i64), P(i32), P(i32)]),
@@ -98,6 +99,7 @@ def lib():
             "ssd_get_hparams": (i32, [vp, P(ssd_hparams), P(C.c_float)]),
             "ssd_set_launch": (i32, [vp, i32, i32]),
             "ssd_set_kernel_shape": (i32, [vp, i32, i32]),
+            "ssd_get_launch": (i32, [vp, P(i32), P(i32), P(i32), P(i32)]),
             "ssd_set_staging": (i32, [vp, i32]),
             "ssd_staging_error": (i32, [vp, P(i32)]),
             "ssd_kernel_launches": (i64, [vp]),
@@ -235,9 +237,19 @@ class Context:
         self._check(lib().ssd_step_tensors(self._h, _ptr_table(grads), first_tensor, num_tensors,
                                            _stream(stream)), "ssd_step_tensors")
 
-    def ssd_step_host(self, host_grads: Sequence, staging: Sequence, host_w_out=None, stream=None):
-        self._check(lib().ssd_step_host(self._h, _ptr_table(host_grads), _ptr_table(staging),
-                                        _ptr(host_w_out), _stream(stream)), "ssd_step_host")
+    def ssd_step_host(self, host_grads: Optional[Sequence], staging: Sequence, host_w_out=None, stream=None):
+        """host_grads None: the gradients are already in `staging` (device memory)."""
+        self._check(lib().ssd_step_host(self._h, None if host_grads is None else _ptr_table(host_grads),
+                                        _ptr_table(staging), _ptr(host_w_out), _stream(stream)), "ssd_step_host")
+
+    def ssd_set_host_chunk(self, chunk_elems: int = 0):
+        self._check(lib().ssd_set_host_chunk(self._h, chunk_elems), "ssd_set_host_chunk")
+
+    def ssd_set_host_pre_weight(self, host_pre, device_slices, slots: int):
+        """host_pre: pinned host tensor / address; device_slices: device tensor / address; (None, None, 0) = off."""
+        self._host_pre = (host_pre, device_slices)       # keep the tensors alive
+        self._check(lib().ssd_set_host_pre_weight(self._h, _ptr(host_pre), _ptr(device_slices), slots),
+                    "ssd_set_host_pre_weight")
 
     def ssd_broadcast_weights(self, stream=None):
         self._check(lib().ssd_broadcast_weights(self._h, _stream(stream)), "ssd_broadcast_weights")
@@ -284,6 +296,12 @@ class Context:
 
     def ssd_set_kernel_shape(self, vector_elems: int = 0, batch: int = 0):
         self._check(lib().ssd_set_kernel_shape(self._h, vector_elems, batch), "ssd_set_kernel_shape")
+
+    def ssd_get_launch(self):
+        """(threads_per_block, blocks_per_sm, vector_elems, batch) overrides, 0 = default"""
+        v = [C.c_int32() for _ in range(4)]
+        self._check(lib().ssd_get_launch(self._h, *[C.byref(x) for x in v]), "ssd_get_launch")
+        return tuple(x.value for x in v)
 
     def ssd_set_staging(self, stages: int = 0):
         self._check(lib().ssd_set_staging(self._h, stages), "ssd_set_staging")

@@ -5,6 +5,7 @@
 #include "ssd_kernels.cuh"
 #include "ssd_ring.cuh"
 
+#include <algorithm>
 #include <cmath>
 #include <cstring>
 #include <map>
@@ -20,12 +21,18 @@ using namespace ssd;
 
 constexpr int64_t kMaxArena = int64_t(1) << 40;
 constexpr int64_t kL2ResidentBytes = 128 << 20;         // a step moving less than this stays within the 126 MB L2
-constexpr int64_t kHostChunkElems = int64_t(1) << 24;   // ssd_step_host: elements per pipelined chunk
+constexpr int64_t kHostChunkElems = int64_t(1) << 24;   // ssd_step_host: default elements per pipelined chunk
+constexpr int kMaxPreSlots = 8;                         // device slices of a host-resident pre_weight
 
 struct Device {
     bool ready = false;
     int id = -1;
     int sms = 0;
+};
+
+// Byte range [lo, hi) of a buffer.
+struct Range {
+    uintptr_t lo, hi;
 };
 
 }  // namespace
@@ -39,6 +46,12 @@ struct ssd_ctx {
     float *w_loc[kMaxWorkers]{}, *pre[kMaxWorkers]{}, *w_dev[kMaxWorkers]{};
     bool has_workers = true;          // false: delay_k == 0 and no worker tables were given
     bool shared_pre = false;          // all K pre_weight pointers are the same buffer
+    bool pre_on_device = true;        // false: created without pre_weight buffers (see ssd_set_host_pre_weight)
+    // pre_weight kept in host memory: one pinned host arena, streamed through `pre_slots` device
+    // slices of `host_chunk` elements by ssd_step_host
+    float *host_pre = nullptr, *pre_slices = nullptr;
+    int pre_slots = 0;
+    int64_t host_chunk = kHostChunkElems;
     int64_t iter = 0, loc_update = 0;
     bool state32 = false;             // every state buffer is 32-byte aligned
     int threads = 0, blocks_per_sm = 0;     // 0: the kernel's default shape
@@ -48,10 +61,12 @@ struct ssd_ctx {
     std::vector<float> lr_mult, wd_mult;
     void *tensor_table = nullptr;
     std::vector<unsigned char> table_image;   // what was last uploaded
+    std::vector<unsigned char> static_image;  // the same for ssd_server_sync_update_static
     // ssd_step_host pipelines chunks over two side streams (copies in, copies out)
     cudaStream_t in_stream = nullptr, out_stream = nullptr;
     std::vector<cudaEvent_t> events;
     std::map<std::pair<const void *, int>, int> occupancy;   // (kernel, threads) -> blocks that fit per SM
+    std::vector<Range> state_ranges;  // the state buffers' byte ranges, sorted by address, free of overlaps
     int64_t launches = 0;
     Device dev;
     std::string cuda_error;
@@ -173,22 +188,25 @@ ssd_status launch(ssd_ctx *c, Kernel kernel, const Params &p, int64_t n, const S
 
 bool aligned32(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 31u) == 0; }
 
-// 8 elements per thread (256-bit accesses) need 32-byte aligned float32 buffers; bfloat16
-// gradient buffers are then read 128 bits at a time and need 16 bytes, which every buffer has.
-bool can_use_256bit(const ssd_ctx *c, bool state32, const void *const *grads, int count)
+// Largest vector a launch may use.  8 elements per thread (256-bit accesses) need 32-byte aligned
+// float32 buffers; bfloat16 gradients are then read 128 bits at a time, which every buffer allows.
+// 16 elements per thread read bfloat16 gradients 256 bits at a time, so those need 32 bytes too.
+// `lo` is the first element of a range launch: it shifts every buffer's alignment.
+int max_vector(const ssd_ctx *c, bool state32, const void *const *grads, int count, int64_t lo,
+               const void *extra = nullptr)
 {
-    if (!state32) return false;
-    if (c->hp.grad_dtype == SSD_F32)
-        for (int i = 0; i < count; ++i)
-            if (!aligned32(grads[i])) return false;
-    return true;
+    if (!state32 || lo % 8 != 0 || (extra && !aligned32(extra))) return 4;
+    bool grads32 = true;
+    for (int i = 0; i < count; ++i) grads32 = grads32 && aligned32(grads[i]);
+    if (c->hp.grad_dtype == SSD_F32) return grads32 ? 16 : 4;
+    return (grads32 && lo % 16 == 0) ? 16 : 8;
 }
 
 // The caller's overrides (ssd_set_kernel_shape, ssd_set_launch) on top of a default shape.
-Shape finish_shape(const ssd_ctx *c, Shape sh, bool wide_ok, int max_batch)
+Shape finish_shape(const ssd_ctx *c, Shape sh, int max_vw, int max_batch)
 {
     if (c->force_vw) sh.vw = c->force_vw;
-    if (sh.vw == 8 && !wide_ok) sh.vw = 4;
+    if (sh.vw > max_vw) sh.vw = max_vw;
     if (c->force_batch) sh.batch = c->force_batch;
     if (sh.batch > max_batch) sh.batch = max_batch;
     if (c->threads) {
@@ -197,6 +215,7 @@ Shape finish_shape(const ssd_ctx *c, Shape sh, bool wide_ok, int max_batch)
     } else if (c->blocks_per_sm) {
         sh.per_sm = c->blocks_per_sm;
     }
+    if (sh.threads > threads_bound(sh.vw)) sh.threads = threads_bound(sh.vw);
     return sh;
 }
 
@@ -205,7 +224,7 @@ Shape finish_shape(const ssd_ctx *c, Shape sh, bool wide_ok, int max_batch)
 // reads and writes: too few bytes in flight cannot cover the DRAM latency, too many lower
 // the DRAM efficiency again, sooner so when a large share of the traffic is writes.  The
 // values below are the measured optima on B200 (arenas of 25M..138M elements).
-Shape sync_shape(const ssd_ctx *c, bool wide_ok)
+Shape sync_shape(const ssd_ctx *c, int max_vw)
 {
     const int K = c->hp.K;
     Shape sh;
@@ -213,25 +232,28 @@ Shape sync_shape(const ssd_ctx *c, bool wide_ok)
         sh = K >= 4 ? Shape{8, 4, 128, 6} : Shape{8, 1, 128, K == 1 ? 4 : 6};
     else
         sh = K >= 4 ? Shape{8, 4, 128, 5} : Shape{8, 1, 128, 6};
-    return finish_shape(c, sh, wide_ok, 8);
+    return finish_shape(c, sh, max_vw, 8);
 }
 
-Shape step_shape(const ssd_ctx *c, int flags, bool wide_ok, int64_t count)
+Shape step_shape(const ssd_ctx *c, int flags, bool shared_pre, int max_vw, int64_t count)
 {
     // Iterations that add K stores per element (pull; refresh or first call with one pre_weight
     // per worker) are write-heavy: 512 threads per SM.  The others: 640 threads per SM.
     const bool sgd = c->hp.local_updater == SSD_LOCAL_SGD;
-    const bool k_extra_stores = (flags & kPull) || (!c->shared_pre && !sgd && (flags & (kRefresh | kFirst)));
+    const bool k_extra_stores = (flags & kPull) || (!shared_pre && !sgd && (flags & (kRefresh | kFirst)));
     Shape sh = k_extra_stores ? Shape{8, 1, 128, 4} : Shape{8, 1, 128, 5};
     // A step whose whole traffic fits in L2 (ResNet-20/56 sized arenas) is bound by latency, not by
     // DRAM: smaller vectors spread it over more threads, and two workers' loads per thread halve the
     // number of dependent round trips.
     const int64_t sg = c->hp.grad_dtype == SSD_BF16 ? 2 : 4;
     if (count * (c->hp.K * (sg + 12) + 16) < kL2ResidentBytes) sh = Shape{4, 2, 64, 0};
-    return finish_shape(c, sh, wide_ok, 4);
+    sh = finish_shape(c, sh, max_vw, 4);
+    // batches that would spill registers under the kernels' thread bounds
+    if (sh.vw >= 8 && sh.batch > 2) sh.batch = 2;
+    return sh;
 }
 
-Shape glu_shape(const ssd_ctx *c, bool wide_ok) { return finish_shape(c, Shape{8, 1, 256, 0}, wide_ok, 1); }
+Shape glu_shape(const ssd_ctx *c, int max_vw) { return finish_shape(c, Shape{8, 1, 256, 0}, max_vw, 1); }
 
 size_t table_end_bytes(const ssd_ctx *c) { return (c->offsets.size() * sizeof(int64_t) + 15) / 16 * 16; }
 size_t table_bytes(const ssd_ctx *c) { return table_end_bytes(c) + c->offsets.size() * sizeof(float4); }
@@ -248,22 +270,31 @@ TensorTable table_of(const ssd_ctx *c)
     return tt;
 }
 
-// Builds the table image from the current hyper-parameters and multipliers and enqueues its
-// upload.  Tensor t: lr*lr_mult[t], wd*wd_mult[t], lr_local*lr_mult[t] (one float multiplication
-// each) and the grad_sync scale of its own lr.
-ssd_status upload_table(ssd_ctx *c, cudaStream_t stream)
+// The per-tensor table as the kernels read it: T tensor ends (int64, padded to 16 bytes), then T
+// float4 {lr, wd, lr_local, c}.  Tensor t: lr*lr_mult[t], wd*wd_mult[t], lr_local*lr_mult[t] (one
+// float multiplication each) and the grad_sync scale of its own lr.  NULL multipliers are all 1.
+void build_table_image(const ssd_ctx *c, const float *lr_mult, const float *wd_mult,
+                       std::vector<unsigned char> *image)
 {
     const size_t T = c->offsets.size();
-    c->table_image.assign(table_bytes(c), 0);
-    int64_t *end = reinterpret_cast<int64_t *>(c->table_image.data());
-    float4 *scal = reinterpret_cast<float4 *>(c->table_image.data() + table_end_bytes(c));
+    image->assign(table_bytes(c), 0);
+    int64_t *end = reinterpret_cast<int64_t *>(image->data());
+    float4 *scal = reinterpret_cast<float4 *>(image->data() + table_end_bytes(c));
     for (size_t t = 0; t < T; ++t) {
         end[t] = t + 1 < T ? c->offsets[t + 1] : c->n;
-        const float lr_t = c->hp.lr * c->lr_mult[t];
-        const float wd_t = c->hp.wd * c->wd_mult[t];
-        const float lr_loc_t = c->hp.lr_local * c->lr_mult[t];
+        const float lm = lr_mult ? lr_mult[t] : 1.0f, wm = wd_mult ? wd_mult[t] : 1.0f;
+        const float lr_t = c->hp.lr * lm;
+        const float wd_t = c->hp.wd * wm;
+        const float lr_loc_t = c->hp.lr_local * lm;
         scal[t] = make_float4(lr_t, wd_t, lr_loc_t, derive_sync_scale(lr_t, c->hp.momentum, c->hp.delay_k));
     }
+}
+
+// Rebuilds the context's table from its current hyper-parameters and multipliers and enqueues
+// the upload into the caller's device table.
+ssd_status upload_table(ssd_ctx *c, cudaStream_t stream)
+{
+    build_table_image(c, c->lr_mult.data(), c->wd_mult.data(), &c->table_image);
     ssd_status st = ensure_device(c);
     if (st != SSD_OK) return st;
     // the image is pageable host memory: the call returns once it has been staged
@@ -273,12 +304,37 @@ ssd_status upload_table(ssd_ctx *c, cudaStream_t stream)
     return SSD_OK;
 }
 
+bool ranges_overlap(const std::vector<Range> &r)      // r sorted by lo
+{
+    for (size_t x = 1; x < r.size(); ++x)
+        if (r[x].lo < r[x - 1].hi) return true;
+    return false;
+}
+
+// A gradient buffer is read-only input: it may not intersect any state buffer (a thread would
+// read what another has already overwritten).  state_ranges is sorted and free of overlaps.
+bool touches_state(const ssd_ctx *c, const void *g, size_t bytes)
+{
+    const uintptr_t lo = reinterpret_cast<uintptr_t>(g), hi = lo + bytes;
+    auto it = std::upper_bound(c->state_ranges.begin(), c->state_ranges.end(), lo,
+                               [](uintptr_t v, const Range &r) { return v < r.hi; });   // first range ending after lo
+    return it != c->state_ranges.end() && it->lo < hi;
+}
+
+size_t grad_bytes(const ssd_ctx *c) { return static_cast<size_t>(c->n) * (c->hp.grad_dtype == SSD_BF16 ? 2 : 4); }
+
+// The GLU rule needs pre_weight; a context created without pre_weight buffers can run its delay
+// stage only through ssd_step_host with a host-resident pre_weight.
+bool lacks_device_pre(const ssd_ctx *c) { return c->hp.local_updater == SSD_LOCAL_GLU && !c->pre_on_device; }
+
 ssd_status check_grads(const ssd_ctx *c, const void *const *grads)
 {
     if (!grads) return SSD_ERR_ARG;
+    const size_t bytes = grad_bytes(c);
     for (int i = 0; i < c->hp.K; ++i) {
         if (!grads[i]) return SSD_ERR_ARG;
         if (!aligned16(grads[i])) return SSD_ERR_ALIGN;
+        if (touches_state(c, grads[i], bytes)) return SSD_ERR_ARG;
     }
     return SSD_OK;
 }
@@ -290,7 +346,9 @@ ssd_status launch_sync_b(ssd_ctx *c, const SyncParams &p, const Shape &sh, cudaS
     case 1: return launch(c, sync_kernel<GT, VW, 1, PT>, p, p.n, sh, stream);
     case 2: return launch(c, sync_kernel<GT, VW, 2, PT>, p, p.n, sh, stream);
     case 4: return launch(c, sync_kernel<GT, VW, 4, PT>, p, p.n, sh, stream);
-    default: return launch(c, sync_kernel<GT, VW, 8, PT>, p, p.n, sh, stream);
+    default:
+        // eight float32 vectors of 16 in flight would spill: four is the most there
+        return launch(c, sync_kernel<GT, VW, (VW == 16 && GT == kF32) ? 4 : 8, PT>, p, p.n, sh, stream);
     }
 }
 
@@ -298,6 +356,8 @@ template <bool PT>
 ssd_status launch_sync_t(ssd_ctx *c, const SyncParams &p, const Shape &sh, cudaStream_t stream)
 {
     const bool bf16 = c->hp.grad_dtype == SSD_BF16;
+    if (sh.vw == 16)
+        return bf16 ? launch_sync_b<kBF16, 16, PT>(c, p, sh, stream) : launch_sync_b<kF32, 16, PT>(c, p, sh, stream);
     if (sh.vw == 8)
         return bf16 ? launch_sync_b<kBF16, 8, PT>(c, p, sh, stream) : launch_sync_b<kF32, 8, PT>(c, p, sh, stream);
     return bf16 ? launch_sync_b<kBF16, 4, PT>(c, p, sh, stream) : launch_sync_b<kF32, 4, PT>(c, p, sh, stream);
@@ -328,8 +388,7 @@ ssd_status launch_sync(ssd_ctx *c, const void *const *grads, int flags, cudaStre
     const bool state32 = (flags & kCopy) ? c->state32 : (aligned32(c->w) && aligned32(c->mom));
     p.tt = table_of(c);
     p.tt.base = lo;
-    // a range that starts 4 elements off an 8-element boundary is only 16-byte aligned
-    const Shape sh = sync_shape(c, lo % 8 == 0 && can_use_256bit(c, state32, grads, c->hp.K));
+    const Shape sh = sync_shape(c, max_vector(c, state32, grads, c->hp.K, lo));
     return p.tt.T ? launch_sync_t<true>(c, p, sh, stream) : launch_sync_t<false>(c, p, sh, stream);
 }
 
@@ -337,6 +396,9 @@ template <bool PT>
 ssd_status launch_glu_t(ssd_ctx *c, const GluParams &p, const Shape &sh, cudaStream_t stream)
 {
     const bool bf16 = c->hp.grad_dtype == SSD_BF16;
+    if (sh.vw == 16)
+        return bf16 ? launch(c, glu_kernel<kBF16, 16, PT>, p, p.n, sh, stream)
+                    : launch(c, glu_kernel<kF32, 16, PT>, p, p.n, sh, stream);
     if (sh.vw == 8)
         return bf16 ? launch(c, glu_kernel<kBF16, 8, PT>, p, p.n, sh, stream)
                     : launch(c, glu_kernel<kF32, 8, PT>, p, p.n, sh, stream);
@@ -349,31 +411,33 @@ ssd_status launch_glu(ssd_ctx *c, int worker, const void *grad, int flags, cudaS
     GluParams p{};
     p.g = grad;
     p.w_loc = c->w_loc[worker];
-    p.pre = c->pre[worker];
+    p.pre = c->pre[worker];                    // NULL only with the plain-SGD updater, which never touches it
     p.w_dev = c->w_dev[worker];
     p.w = c->w;
     p.n = c->n;
     p.flags = flags | (c->hp.local_updater == SSD_LOCAL_SGD ? kLocalSgd : 0);
     p.s = c->s;
     p.tt = table_of(c);
-    const Shape sh = glu_shape(c, can_use_256bit(c, c->state32, &grad, 1));
+    const Shape sh = glu_shape(c, max_vector(c, c->state32, &grad, 1, 0));
     return p.tt.T ? launch_glu_t<true>(c, p, sh, stream) : launch_glu_t<false>(c, p, sh, stream);
 }
 
 template <int GT, int VW, bool PT>
 ssd_status launch_step_b(ssd_ctx *c, const StepParams &p, const Shape &sh, cudaStream_t stream)
 {
-    switch (sh.batch) {
-    case 1: return launch(c, step_kernel<GT, VW, 1, PT>, p, p.n, sh, stream);
-    case 2: return launch(c, step_kernel<GT, VW, 2, PT>, p, p.n, sh, stream);
-    default: return launch(c, step_kernel<GT, VW, 4, PT>, p, p.n, sh, stream);
-    }
+    // step_shape keeps the batch at 2 or below for vectors of 8 and more (4 would spill)
+    if (sh.batch == 1) return launch(c, step_kernel<GT, VW, 1, PT>, p, p.n, sh, stream);
+    if constexpr (VW == 4)
+        if (sh.batch > 2) return launch(c, step_kernel<GT, 4, 4, PT>, p, p.n, sh, stream);
+    return launch(c, step_kernel<GT, VW, 2, PT>, p, p.n, sh, stream);
 }
 
 template <bool PT>
 ssd_status launch_step_t(ssd_ctx *c, const StepParams &p, const Shape &sh, cudaStream_t stream)
 {
     const bool bf16 = c->hp.grad_dtype == SSD_BF16;
+    if (sh.vw == 16)
+        return bf16 ? launch_step_b<kBF16, 16, PT>(c, p, sh, stream) : launch_step_b<kF32, 16, PT>(c, p, sh, stream);
     if (sh.vw == 8)
         return bf16 ? launch_step_b<kBF16, 8, PT>(c, p, sh, stream) : launch_step_b<kF32, 8, PT>(c, p, sh, stream);
     return bf16 ? launch_step_b<kBF16, 4, PT>(c, p, sh, stream) : launch_step_b<kF32, 4, PT>(c, p, sh, stream);
@@ -382,9 +446,9 @@ ssd_status launch_step_t(ssd_ctx *c, const StepParams &p, const Shape &sh, cudaS
 // The shared-memory ring covers the common case; the rest stays on the register path.  Its bulk
 // copies need 16-byte aligned sources and sizes, which bfloat16 gradients give only for ranges that
 // start and end on multiples of 8 elements.
-bool ring_can_run(const ssd_ctx *c, int64_t lo, int64_t count)
+bool ring_can_run(const ssd_ctx *c, bool shared_pre, int64_t lo, int64_t count)
 {
-    if (c->shared_pre || c->hp.local_updater != SSD_LOCAL_GLU) return false;
+    if (shared_pre || c->hp.local_updater != SSD_LOCAL_GLU) return false;
     if (c->hp.grad_dtype == SSD_BF16 && (lo % 8 != 0 || count % 8 != 0)) return false;
     return true;
 }
@@ -417,14 +481,18 @@ ssd_status launch_step_ring(ssd_ctx *c, const StepParams &p, cudaStream_t stream
                 : launch_ring(c, step_ring_kernel<kF32, false>, p, stream);
 }
 
+// pre_slice: when not NULL, the one pre_weight of all workers for exactly this range, at
+// pre_slice[0 .. count) (a device slice of a host-resident pre_weight); the context's own
+// pre_weight pointers are then not used.
 ssd_status launch_step(ssd_ctx *c, const void *const *grads, int flags, cudaStream_t stream,
-                       int64_t lo = 0, int64_t count = -1)
+                       int64_t lo = 0, int64_t count = -1, float *pre_slice = nullptr)
 {
     StepParams p{};
+    const bool shared = c->shared_pre || pre_slice;
     for (int i = 0; i < c->hp.K; ++i) {
         p.g[i] = grad_at(c, grads[i], lo);
         p.w_loc[i] = c->w_loc[i] + lo;
-        p.pre[i] = c->pre[i] + lo;
+        p.pre[i] = pre_slice ? pre_slice : c->pre[i] ? c->pre[i] + lo : nullptr;
         p.w_dev[i] = c->w_dev[i] + lo;
     }
     p.w = c->w + lo;
@@ -432,12 +500,12 @@ ssd_status launch_step(ssd_ctx *c, const void *const *grads, int flags, cudaStre
     p.n = count < 0 ? c->n : count;
     p.K = c->hp.K;
     p.flags = flags | (c->hp.local_updater == SSD_LOCAL_SGD ? kLocalSgd : 0);
-    p.shared_pre = c->shared_pre ? 1 : 0;
+    p.shared_pre = shared ? 1 : 0;
     p.s = c->s;
     p.tt = table_of(c);
     p.tt.base = lo;
-    if (c->staging && ring_can_run(c, lo, p.n)) return launch_step_ring(c, p, stream);
-    const Shape sh = step_shape(c, flags, lo % 8 == 0 && can_use_256bit(c, c->state32, grads, c->hp.K), p.n);
+    if (c->staging && ring_can_run(c, shared, lo, p.n)) return launch_step_ring(c, p, stream);
+    const Shape sh = step_shape(c, flags, shared, max_vector(c, c->state32, grads, c->hp.K, lo, pre_slice), p.n);
     return p.tt.T ? launch_step_t<true>(c, p, sh, stream) : launch_step_t<false>(c, p, sh, stream);
 }
 
@@ -448,7 +516,7 @@ ssd_status launch_copy(ssd_ctx *c, int first_worker, int count, cudaStream_t str
     p.src = c->w;
     p.n = c->n;
     p.K = count;
-    const Shape sh = finish_shape(c, Shape{8, 1, 256, 0}, c->state32, 1);
+    Shape sh = finish_shape(c, Shape{8, 1, 256, 0}, c->state32 ? 8 : 4, 1);
     if (sh.vw == 8) return launch(c, copy_kernel<8>, p, p.n, sh, stream);
     return launch(c, copy_kernel<4>, p, p.n, sh, stream);
 }
@@ -463,13 +531,13 @@ void advance(ssd_ctx *c)
 
 // ---------------------------------------------------------------------------
 // Per-tensor table in static device memory, for ssd_server_sync_update_static.
-// Layout: SSD_STATIC_TABLE_MAX_TENSORS tensor ends (int64), then as many float4
-// {lr, wd, lr_local, c}.  Every GPU that loads this library holds the 24 KB until
-// the process exits.  In host code the name below is only a handle for
-// cudaGetSymbolAddress; kernels get the device address that call returns.
+// Same layout as the caller-allocated table (T tensor ends padded to 16 bytes, then T
+// float4 {lr, wd, lr_local, c}), sized for SSD_STATIC_TABLE_MAX_TENSORS tensors.
+// Every GPU that loads this library holds the 24 KB until the process exits.  In
+// host code the name below is only a handle for cudaGetSymbolAddress; kernels get
+// the device address that call returns.
 // ---------------------------------------------------------------------------
-constexpr size_t kStaticEndBytes = SSD_STATIC_TABLE_MAX_TENSORS * sizeof(int64_t);
-constexpr size_t kStaticTableBytes = kStaticEndBytes + SSD_STATIC_TABLE_MAX_TENSORS * sizeof(float4);
+constexpr size_t kStaticTableBytes = SSD_STATIC_TABLE_MAX_TENSORS * (sizeof(int64_t) + sizeof(float4));
 static __device__ __align__(256) unsigned char g_static_tensor_table[kStaticTableBytes];
 
 constexpr int kMaxDevices = 64;
@@ -521,9 +589,12 @@ ssd_status ssd_init(ssd_ctx **out, const ssd_layout *layout, const ssd_hparams *
         std::isinf(hp->rescale))
         return SSD_ERR_ARG;
     // Without a delay stage (delay_k == 0) no worker state is ever touched: the tables may be NULL.
-    const bool workers = hp->delay_k > 0 || (b->w_loc && b->pre && b->w_dev);
+    // A NULL `pre` table with worker state means that pre_weight does not live in device memory
+    // (ssd_set_host_pre_weight), or is never used (plain-SGD local updater).
+    const bool workers = b->w_loc && b->w_dev && (hp->delay_k > 0 || b->pre);
+    const bool device_pre = workers && b->pre;
     if (!b->w || !b->mom) return SSD_ERR_ARG;
-    if (hp->delay_k > 0 && (!b->w_loc || !b->pre || !b->w_dev)) return SSD_ERR_ARG;
+    if (hp->delay_k > 0 && (!b->w_loc || !b->w_dev)) return SSD_ERR_ARG;
 
     ssd_ctx *c = new (std::nothrow) ssd_ctx;
     if (!c) return SSD_ERR_NOMEM;
@@ -534,23 +605,27 @@ ssd_status ssd_init(ssd_ctx **out, const ssd_layout *layout, const ssd_hparams *
     }
     // All K pre_weight pointers equal: one shared pre_weight (its K copies always hold the same
     // values, every worker takes it from the same pulled global weight).
-    bool shared_pre = workers && hp->K > 1 && b->pre[0] != nullptr;
+    bool shared_pre = device_pre && hp->K > 1 && b->pre[0] != nullptr;
     for (int i = 1; shared_pre && i < hp->K; ++i) shared_pre = b->pre[i] == b->pre[0];
     std::vector<const void *> all{b->w, b->mom};
     for (int i = 0; workers && i < hp->K; ++i) {
         all.push_back(b->w_loc[i]);
-        if (!shared_pre || i == 0) all.push_back(b->pre[i]);
+        if (device_pre && (!shared_pre || i == 0)) all.push_back(b->pre[i]);
         all.push_back(b->w_dev[i]);
     }
     for (const void *p : all) {
         if (!p) st = SSD_ERR_ARG;
         else if (!aligned16(p) && st == SSD_OK) st = SSD_ERR_ALIGN;
     }
-    // No two state buffers may share an address: every element is read and written
-    // by one thread only, which holds only if the buffers are distinct.
-    for (size_t x = 0; x < all.size() && st == SSD_OK; ++x)
-        for (size_t y = x + 1; y < all.size(); ++y)
-            if (all[x] == all[y]) st = SSD_ERR_ARG;
+    // No two state buffers may overlap: every element is read and written by one thread only,
+    // which holds only if the buffers are disjoint.
+    const size_t arena_bytes = static_cast<size_t>(c->n) * sizeof(float);
+    for (const void *p : all) {
+        const uintptr_t lo = reinterpret_cast<uintptr_t>(p);
+        c->state_ranges.push_back(Range{lo, lo + arena_bytes});
+    }
+    std::sort(c->state_ranges.begin(), c->state_ranges.end(), [](const Range &x, const Range &y) { return x.lo < y.lo; });
+    if (st == SSD_OK && ranges_overlap(c->state_ranges)) st = SSD_ERR_ARG;
     if (st != SSD_OK) {
         delete c;
         return st;
@@ -573,11 +648,12 @@ ssd_status ssd_init(ssd_ctx **out, const ssd_layout *layout, const ssd_hparams *
     c->mom = b->mom;
     c->has_workers = workers;
     c->shared_pre = shared_pre;
+    c->pre_on_device = device_pre;
     c->state32 = true;
     for (const void *p : all) c->state32 = c->state32 && aligned32(p);
     for (int i = 0; workers && i < hp->K; ++i) {
         c->w_loc[i] = b->w_loc[i];
-        c->pre[i] = b->pre[i];
+        c->pre[i] = device_pre ? b->pre[i] : nullptr;
         c->w_dev[i] = b->w_dev[i];
     }
     *out = c;
@@ -630,28 +706,22 @@ ssd_status ssd_server_sync_update_static(ssd_ctx *ctx, const void *const *grads,
     }
     st = ensure_device(ctx);
     if (st != SSD_OK) return st;
+    // the array's address differs per device: the context's device must be the current one
+    int current = -1;
+    cudaError_t e = cudaGetDevice(&current);
+    if (e != cudaSuccess) return cuda_fail(ctx, e);
+    if (current != ctx->dev.id) return SSD_ERR_STATE;
     unsigned char *table = nullptr;
     st = static_table_address(ctx, &table);
     if (st != SSD_OK) return st;
 
-    // Same per-tensor scalars as ssd_set_tensor_scales derives, written over the first T
-    // entries of the static table; entries beyond T keep older contents and are never read.
-    std::vector<int64_t> end(T);
-    std::vector<float4> scal(T);
-    for (size_t t = 0; t < T; ++t) {
-        end[t] = t + 1 < T ? ctx->offsets[t + 1] : ctx->n;
-        const float lm = lr_mult ? lr_mult[t] : 1.0f, wm = wd_mult ? wd_mult[t] : 1.0f;
-        const float lr_t = ctx->hp.lr * lm;
-        const float wd_t = ctx->hp.wd * wm;
-        const float lr_loc_t = ctx->hp.lr_local * lm;
-        scal[t] = make_float4(lr_t, wd_t, lr_loc_t, derive_sync_scale(lr_t, ctx->hp.momentum, ctx->hp.delay_k));
-    }
+    // The image ssd_set_tensor_scales would upload, built by the same code and kept in the
+    // context until the next call replaces it, written over the front of the static array
+    // (bytes beyond it keep older contents and are never read).
+    build_table_image(ctx, lr_mult, wd_mult, &ctx->static_image);
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    // pageable sources: each call returns once its bytes have been staged
-    cudaError_t e = cudaMemcpyAsync(table, end.data(), T * sizeof(int64_t), cudaMemcpyHostToDevice, stream);
-    if (e == cudaSuccess)
-        e = cudaMemcpyAsync(table + kStaticEndBytes, scal.data(), T * sizeof(float4), cudaMemcpyHostToDevice,
-                            stream);
+    // pageable source: the call returns once the bytes have been staged
+    e = cudaMemcpyAsync(table, ctx->static_image.data(), ctx->static_image.size(), cudaMemcpyHostToDevice, stream);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
 
     SyncParams p{};
@@ -663,10 +733,10 @@ ssd_status ssd_server_sync_update_static(ssd_ctx *ctx, const void *const *grads,
     p.flags = 0;
     p.s = ctx->s;
     p.tt.end = reinterpret_cast<const int64_t *>(table);
-    p.tt.scal = reinterpret_cast<const float4 *>(table + kStaticEndBytes);
+    p.tt.scal = reinterpret_cast<const float4 *>(table + table_end_bytes(ctx));
     p.tt.T = static_cast<int>(T);
     const bool state32 = aligned32(ctx->w) && aligned32(ctx->mom);
-    const Shape sh = sync_shape(ctx, can_use_256bit(ctx, state32, grads, ctx->hp.K));
+    const Shape sh = sync_shape(ctx, max_vector(ctx, state32, grads, ctx->hp.K, 0));
     return launch_sync_t<true>(ctx, p, sh, stream);
 }
 
@@ -677,8 +747,9 @@ ssd_status ssd_worker_glu_update(ssd_ctx *ctx, int32_t worker, const void *grad,
     if (worker < 0 || worker >= ctx->hp.K) return SSD_ERR_ARG;
     if (flags & ~(SSD_FLAG_FIRST | SSD_FLAG_REFRESH | SSD_FLAG_PULL)) return SSD_ERR_ARG;
     if (ctx->hp.delay_k == 0) return SSD_ERR_STATE;
-    if (ctx->shared_pre) return SSD_ERR_STATE;
+    if (ctx->shared_pre || lacks_device_pre(ctx)) return SSD_ERR_STATE;
     if (!aligned16(grad)) return SSD_ERR_ALIGN;
+    if (touches_state(ctx, grad, grad_bytes(ctx))) return SSD_ERR_ARG;
     return launch_glu(ctx, worker, grad, flags, static_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -694,8 +765,9 @@ ssd_status ssd_worker_local_step(ssd_ctx *ctx, int32_t worker, const void *grad,
         return SSD_OK;
     }
     if (!grad) return SSD_ERR_ARG;
-    if (ctx->shared_pre) return SSD_ERR_STATE;
+    if (ctx->shared_pre || lacks_device_pre(ctx)) return SSD_ERR_STATE;
     if (!aligned16(grad)) return SSD_ERR_ALIGN;
+    if (touches_state(ctx, grad, grad_bytes(ctx))) return SSD_ERR_ARG;
     return launch_glu(ctx, worker, grad, flags, stream);
 }
 
@@ -713,6 +785,7 @@ ssd_status ssd_step(ssd_ctx *ctx, const void *const *grads, void *cuda_stream)
     if (st != SSD_OK) return st;
     int32_t stage, flags;
     schedule_of(ctx, ctx->iter, &stage, &flags);
+    if (stage == SSD_STAGE_DELAY && lacks_device_pre(ctx)) return SSD_ERR_STATE;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     st = (stage == SSD_STAGE_WARMUP) ? launch_sync(ctx, grads, flags & SSD_FLAG_COPY, stream)
                                      : launch_step(ctx, grads, flags, stream);
@@ -734,6 +807,7 @@ ssd_status ssd_step_tensors(ssd_ctx *ctx, const void *const *grads, int32_t firs
     if (hi == lo) return SSD_OK;                      // only empty tensors
     int32_t stage, flags;
     schedule_of(ctx, ctx->iter, &stage, &flags);
+    if (stage == SSD_STAGE_DELAY && lacks_device_pre(ctx)) return SSD_ERR_STATE;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     return (stage == SSD_STAGE_WARMUP) ? launch_sync(ctx, grads, flags & SSD_FLAG_COPY, stream, lo, hi - lo)
                                        : launch_step(ctx, grads, flags, stream, lo, hi - lo);
@@ -742,69 +816,124 @@ ssd_status ssd_step_tensors(ssd_ctx *ctx, const void *const *grads, int32_t firs
 ssd_status ssd_step_host(ssd_ctx *ctx, const void *const *host_grads, void *const *staging,
                          float *host_w_out, void *cuda_stream)
 {
-    if (!ctx || !host_grads || !staging) return SSD_ERR_ARG;
+    if (!ctx || !staging) return SSD_ERR_ARG;
     for (int i = 0; i < ctx->hp.K; ++i) {
-        if (!host_grads[i] || !staging[i]) return SSD_ERR_ARG;
+        if (!staging[i] || (host_grads && !host_grads[i])) return SSD_ERR_ARG;
         if (!aligned16(staging[i])) return SSD_ERR_ALIGN;
+        if (touches_state(ctx, staging[i], grad_bytes(ctx))) return SSD_ERR_ARG;
     }
+    int32_t stage, flags;
+    schedule_of(ctx, ctx->iter, &stage, &flags);
+    const bool glu_stage = stage == SSD_STAGE_DELAY && ctx->hp.local_updater == SSD_LOCAL_GLU;
+    if (glu_stage && !ctx->pre_on_device && !ctx->host_pre) return SSD_ERR_STATE;
     ssd_status st = ensure_device(ctx);
     if (st != SSD_OK) return st;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const int K = ctx->hp.K;
     const size_t sg = ctx->hp.grad_dtype == SSD_BF16 ? 2 : 4;
-    int32_t stage, flags;
-    schedule_of(ctx, ctx->iter, &stage, &flags);
+    // A host-resident pre_weight travels with the gradients: its slice of a chunk is copied into
+    // one of the device slices before the chunk's kernel (not on the first GLU call, which does
+    // not read it) and copied back after it on the iterations that overwrite it.
+    const bool host_pre = glu_stage && ctx->host_pre;
+    const bool pre_in = host_pre && !(flags & SSD_FLAG_FIRST);
+    const bool pre_out = host_pre && (flags & (SSD_FLAG_FIRST | SSD_FLAG_REFRESH));
+    const int slots = ctx->pre_slots;
 
-    // The arena is cut into chunks; chunk c's gradients are copied in on a side stream while
-    // chunk c-1 is being updated on the caller's stream and chunk c-2's new weights are copied
+    // The arena is cut into chunks; chunk c's inputs are copied in on a side stream while
+    // chunk c-1 is being updated on the caller's stream and chunk c-2's results are copied
     // out on a second side stream.  The update is elementwise, so chunks are independent.
-    const int64_t chunk = kHostChunkElems;
+    const int64_t chunk = ctx->host_chunk;
     const int chunks = static_cast<int>((ctx->n + chunk - 1) / chunk);
+    // events: [2c] chunk c copied in, [2c+1] chunk c updated, then start, end, and one per device
+    // slice ("the slice may be overwritten")
+    const size_t ev_start_at = 2 * static_cast<size_t>(chunks), ev_end_at = ev_start_at + 1, ev_slot_at = ev_start_at + 2;
     cudaError_t e = cudaSuccess;
     if (!ctx->in_stream) e = cudaStreamCreateWithFlags(&ctx->in_stream, cudaStreamNonBlocking);
     if (e == cudaSuccess && !ctx->out_stream) e = cudaStreamCreateWithFlags(&ctx->out_stream, cudaStreamNonBlocking);
-    while (e == cudaSuccess && ctx->events.size() < static_cast<size_t>(2 * chunks + 2)) {
+    while (e == cudaSuccess && ctx->events.size() < ev_slot_at + kMaxPreSlots) {
         cudaEvent_t ev;
         e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
         if (e == cudaSuccess) ctx->events.push_back(ev);
     }
     if (e != cudaSuccess) return cuda_fail(ctx, e);
-    cudaEvent_t ev_start = ctx->events[2 * chunks], ev_end = ctx->events[2 * chunks + 1];
+    cudaEvent_t ev_start = ctx->events[ev_start_at], ev_end = ctx->events[ev_end_at];
+    const bool copies_out = host_w_out || pre_out;
     // everything already enqueued on the caller's stream comes first
     e = cudaEventRecord(ev_start, stream);
     if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->in_stream, ev_start, 0);
-    if (e == cudaSuccess && host_w_out) e = cudaStreamWaitEvent(ctx->out_stream, ev_start, 0);
+    if (e == cudaSuccess && copies_out) e = cudaStreamWaitEvent(ctx->out_stream, ev_start, 0);
     if (e != cudaSuccess) return cuda_fail(ctx, e);
     for (int c = 0; c < chunks; ++c) {
         const int64_t lo = static_cast<int64_t>(c) * chunk;
         const int64_t count = ctx->n - lo < chunk ? ctx->n - lo : chunk;
-        for (int i = 0; i < K && e == cudaSuccess; ++i)
+        const int slot = host_pre ? c % slots : 0;
+        float *slice = host_pre ? ctx->pre_slices + static_cast<int64_t>(slot) * chunk : nullptr;
+        cudaEvent_t ev_slot = ctx->events[ev_slot_at + slot];
+        // the slice is free once the chunk that used it last (c - slots) is done with it
+        if (host_pre && c >= slots) e = cudaStreamWaitEvent(ctx->in_stream, ev_slot, 0);
+        for (int i = 0; host_grads && i < K && e == cudaSuccess; ++i)
             e = cudaMemcpyAsync(static_cast<unsigned char *>(staging[i]) + lo * sg,
                                 static_cast<const unsigned char *>(host_grads[i]) + lo * sg, count * sg,
                                 cudaMemcpyHostToDevice, ctx->in_stream);
+        if (e == cudaSuccess && pre_in)
+            e = cudaMemcpyAsync(slice, ctx->host_pre + lo, count * sizeof(float), cudaMemcpyHostToDevice,
+                                ctx->in_stream);
         if (e == cudaSuccess) e = cudaEventRecord(ctx->events[2 * c], ctx->in_stream);
         if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, ctx->events[2 * c], 0);
         if (e != cudaSuccess) return cuda_fail(ctx, e);
         st = (stage == SSD_STAGE_WARMUP)
                  ? launch_sync(ctx, const_cast<const void *const *>(staging), flags & SSD_FLAG_COPY, stream, lo, count)
-                 : launch_step(ctx, const_cast<const void *const *>(staging), flags, stream, lo, count);
+                 : launch_step(ctx, const_cast<const void *const *>(staging), flags, stream, lo, count, slice);
         if (st != SSD_OK) return st;
-        if (host_w_out) {
+        if (copies_out) {
             e = cudaEventRecord(ctx->events[2 * c + 1], stream);
             if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->out_stream, ctx->events[2 * c + 1], 0);
-            if (e == cudaSuccess)
+            if (e == cudaSuccess && host_w_out)
                 e = cudaMemcpyAsync(host_w_out + lo, ctx->w + lo, count * sizeof(float), cudaMemcpyDeviceToHost,
                                     ctx->out_stream);
-            if (e != cudaSuccess) return cuda_fail(ctx, e);
+            if (e == cudaSuccess && pre_out)
+                e = cudaMemcpyAsync(ctx->host_pre + lo, slice, count * sizeof(float), cudaMemcpyDeviceToHost,
+                                    ctx->out_stream);
         }
+        if (e == cudaSuccess && host_pre) e = cudaEventRecord(ev_slot, pre_out ? ctx->out_stream : stream);
+        if (e != cudaSuccess) return cuda_fail(ctx, e);
     }
-    if (host_w_out) {
+    if (copies_out) {
         // the caller's stream ends behind the last copy out
         e = cudaEventRecord(ev_end, ctx->out_stream);
         if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, ev_end, 0);
         if (e != cudaSuccess) return cuda_fail(ctx, e);
     }
     advance(ctx);
+    return SSD_OK;
+}
+
+ssd_status ssd_set_host_chunk(ssd_ctx *ctx, int64_t chunk_elems)
+{
+    if (!ctx) return SSD_ERR_ARG;
+    if (chunk_elems == 0) chunk_elems = kHostChunkElems;
+    if (chunk_elems < 1024 || chunk_elems % 1024 != 0 || chunk_elems > (int64_t(1) << 30)) return SSD_ERR_ARG;
+    if (ctx->host_pre) return SSD_ERR_STATE;          // the device slices were sized for the current chunk
+    ctx->host_chunk = chunk_elems;
+    return SSD_OK;
+}
+
+ssd_status ssd_set_host_pre_weight(ssd_ctx *ctx, float *host_pre, float *device_slices, int32_t slots)
+{
+    if (!ctx) return SSD_ERR_ARG;
+    if (!host_pre && !device_slices && slots == 0) {       // off again
+        ctx->host_pre = ctx->pre_slices = nullptr;
+        ctx->pre_slots = 0;
+        return SSD_OK;
+    }
+    if (!host_pre || !device_slices || slots < 1 || slots > kMaxPreSlots) return SSD_ERR_ARG;
+    if (!ctx->has_workers || ctx->hp.delay_k == 0 || ctx->pre_on_device) return SSD_ERR_STATE;
+    if (!aligned16(host_pre) || !aligned16(device_slices)) return SSD_ERR_ALIGN;
+    const size_t bytes = static_cast<size_t>(slots) * static_cast<size_t>(ctx->host_chunk) * sizeof(float);
+    if (touches_state(ctx, device_slices, bytes)) return SSD_ERR_ARG;
+    ctx->host_pre = host_pre;
+    ctx->pre_slices = device_slices;
+    ctx->pre_slots = slots;
     return SSD_OK;
 }
 
@@ -928,15 +1057,26 @@ ssd_status ssd_set_launch(ssd_ctx *ctx, int32_t threads_per_block, int32_t block
         (threads_per_block < 64 || threads_per_block > kMaxThreads || threads_per_block % 32 != 0))
         return SSD_ERR_ARG;
     if (blocks_per_sm < 0 || blocks_per_sm > 32) return SSD_ERR_ARG;
-    if (threads_per_block) ctx->threads = threads_per_block;
+    ctx->threads = threads_per_block;
     ctx->blocks_per_sm = blocks_per_sm;
+    return SSD_OK;
+}
+
+ssd_status ssd_get_launch(const ssd_ctx *ctx, int32_t *threads_per_block, int32_t *blocks_per_sm,
+                          int32_t *vector_elems, int32_t *batch)
+{
+    if (!ctx) return SSD_ERR_ARG;
+    if (threads_per_block) *threads_per_block = ctx->threads;
+    if (blocks_per_sm) *blocks_per_sm = ctx->blocks_per_sm;
+    if (vector_elems) *vector_elems = ctx->force_vw;
+    if (batch) *batch = ctx->force_batch;
     return SSD_OK;
 }
 
 ssd_status ssd_set_kernel_shape(ssd_ctx *ctx, int32_t vector_elems, int32_t batch)
 {
     if (!ctx) return SSD_ERR_ARG;
-    if (vector_elems != 0 && vector_elems != 4 && vector_elems != 8) return SSD_ERR_ARG;
+    if (vector_elems != 0 && vector_elems != 4 && vector_elems != 8 && vector_elems != 16) return SSD_ERR_ARG;
     if (batch != 0 && batch != 1 && batch != 2 && batch != 4 && batch != 8) return SSD_ERR_ARG;
     ctx->force_vw = vector_elems;
     ctx->force_batch = batch;
@@ -970,7 +1110,7 @@ const char *ssd_status_str(ssd_status status)
     case SSD_ERR_ARG: return "invalid argument";
     case SSD_ERR_ALIGN: return "device pointer not 16-byte aligned";
     case SSD_ERR_LAYOUT: return "invalid parameter layout";
-    case SSD_ERR_STATE: return "call not valid in the current stage";
+    case SSD_ERR_STATE: return "call not valid in the context's current stage or mode";
     case SSD_ERR_CUDA: return "CUDA runtime error";
     case SSD_ERR_NOMEM: return "out of host memory";
     case SSD_ERR_TOO_LARGE: return "more tensors than the static table holds (SSD_STATIC_TABLE_MAX_TENSORS)";

@@ -19,7 +19,10 @@ def bits(a):
     return np.ascontiguousarray(a).view(np.uint32)
 
 
-def assert_same(got, want, what, idx=None):
+def assert_same(got, want, what, idx=None, generated_nans=False):
+    """Bit equality of every element.  generated_nans: where the oracle's value is a NaN that the
+    arithmetic produced (inf - inf, 0 * inf), only "is a NaN" is compared: IEEE 754 leaves the sign
+    and payload of such a NaN open, and x86 and the GPU choose differently."""
     if isinstance(got, torch.Tensor):
         if idx is not None:                       # gather on the device: the arena may be GiB-sized
             got = got[torch.from_numpy(np.asarray(idx)).to(got.device)]
@@ -30,6 +33,10 @@ def assert_same(got, want, what, idx=None):
     if idx is not None:
         g = g[idx]
     gb, wb = bits(g), bits(want)
+    if generated_nans:
+        nan = np.isnan(want)
+        assert np.array_equal(np.isnan(g), nan), f"{what}: NaNs in different places"
+        gb, wb = np.where(nan, 0, gb), np.where(nan, 0, wb)
     if not np.array_equal(gb, wb):
         bad = np.nonzero(gb != wb)[0]
         j = int(bad[0])
@@ -60,13 +67,17 @@ def oracle_grad(g: torch.Tensor, bf16: bool):
     return g.detach().cpu().numpy()
 
 
-def compare_states(dev: DeviceState, ref: oracle.State, tag, idx=None):
-    assert_same(dev.w, ref.w, f"{tag} w", idx)
-    assert_same(dev.mom, ref.mom, f"{tag} mom", idx)
+def compare_states(dev: DeviceState, ref: oracle.State, tag, idx=None, generated_nans=False):
+    kw = dict(idx=idx, generated_nans=generated_nans)
+    assert_same(dev.w, ref.w, f"{tag} w", **kw)
+    assert_same(dev.mom, ref.mom, f"{tag} mom", **kw)
     for i in range(dev.K):
-        assert_same(dev.w_loc[i], ref.w_loc[i], f"{tag} w_loc[{i}]", idx)
-        assert_same(dev.pre[i], ref.pre[i], f"{tag} pre[{i}]", idx)
-        assert_same(dev.w_dev[i], ref.w_dev[i], f"{tag} w_dev[{i}]", idx)
+        assert_same(dev.w_loc[i], ref.w_loc[i], f"{tag} w_loc[{i}]", **kw)
+        assert_same(dev.pre[i], ref.pre[i], f"{tag} pre[{i}]", **kw)
+        assert_same(dev.w_dev[i], ref.w_dev[i], f"{tag} w_dev[{i}]", **kw)
+    # nothing was stored outside the arenas (guard words before, between and after them)
+    for slab in getattr(dev, "slabs", []):
+        assert slab.guards_intact(), f"{tag}: guard words overwritten next to arenas {slab.damaged_gaps()}"
     it, lu, _, _ = dev.ctx.ssd_get_counters()
     assert (it, lu) == (ref.iter, ref.loc_update), tag
     for i in range(dev.K):

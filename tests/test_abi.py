@@ -245,3 +245,117 @@ def test_header_is_valid_c_and_cpp(tmp_path):
                            "-c", str(c), "-o", str(tmp_path / "use_c.o")])
     subprocess.check_call(["g++", "-std=c++11", "-Wall", "-Werror", "-I", os.path.dirname(header), "-x", "c++",
                            "-c", str(c), "-o", str(tmp_path / "use_cpp.o")])
+
+
+def test_launch_overrides_are_set_and_reset_together():
+    ctx = make_ctx()
+    assert ctx.ssd_get_launch() == (0, 0, 0, 0)
+    ctx.ssd_set_launch(256, 3)
+    ctx.ssd_set_kernel_shape(16, 2)
+    assert ctx.ssd_get_launch() == (256, 3, 16, 2)
+    ctx.ssd_set_launch(0, 5)                       # 0 returns the thread count to the default
+    assert ctx.ssd_get_launch() == (0, 5, 16, 2)
+    ctx.ssd_set_launch(128, 0)
+    assert ctx.ssd_get_launch() == (128, 0, 16, 2)
+    ctx.ssd_set_launch()
+    ctx.ssd_set_kernel_shape()
+    assert ctx.ssd_get_launch() == (0, 0, 0, 0)
+    with pytest.raises(B.SsdError):
+        ctx.ssd_set_kernel_shape(32, 1)
+
+
+def test_overlapping_buffers_are_rejected():
+    K = 2
+    hp = B.make_hparams(K, 0.1, 0.9, 2, 4)
+    n = 1 << 20                                               # 4 MiB arenas
+    w, mom, wl, pre, wdv = fake_ptrs(K, step=n * 4)           # back to back: allowed
+    B.Context([n], hp, w, mom, wl, pre, wdv)
+    for shift in (16, n * 4 - 16):                            # slices of one slab with a wrong stride
+        with pytest.raises(B.SsdError) as e:
+            B.Context([n], hp, w, mom + shift - n * 4, wl, pre, wdv)
+        assert e.value.status == B.SSD_ERR_ARG
+        with pytest.raises(B.SsdError) as e:
+            B.Context([n], hp, w, mom, wl, pre, [wdv[0], wl[0] + shift])
+        assert e.value.status == B.SSD_ERR_ARG
+    ctx = B.Context([n], hp, w, mom, wl, pre, wdv)
+    free = wdv[-1] + n * 4
+    ok = [free, free + n * 4]
+    inside = [[w + 64, ok[1]], [ok[0], pre[1] - 32], [wdv[1] + n * 4 - 16, ok[1]], [ok[0], w - n * 4 + 16]]
+    for grads in inside:                                      # a gradient range that reaches into the state
+        for call in (ctx.ssd_step, ctx.ssd_server_sync_update):
+            with pytest.raises(B.SsdError) as e:
+                call(grads)
+            assert e.value.status == B.SSD_ERR_ARG
+    assert ctx.ssd_kernel_launches() == 0 and ctx.ssd_get_counters()[0] == 0
+    ctx0 = B.Context([n], B.make_hparams(K, 0.1, 0.9, 0, 4), w, mom, wl, pre, wdv)
+    with pytest.raises(B.SsdError) as e:
+        ctx0.ssd_worker_glu_update(0, mom + 4096, 0)
+    assert e.value.status == B.SSD_ERR_ARG
+    # bfloat16 gradient arenas are half as long: the same start address may be free of the state
+    hp16 = B.make_hparams(K, 0.1, 0.9, 2, 4, grad_dtype=B.SSD_BF16)
+    ctx16 = B.Context([n], hp16, w, mom, wl, pre, wdv)
+    with pytest.raises(B.SsdError) as e:
+        ctx16.ssd_server_sync_update([w - n * 2 + 16, ok[0]])
+    assert e.value.status == B.SSD_ERR_ARG
+
+
+def test_host_pre_weight_mode_is_validated():
+    K, n = 2, 4096
+    hp = B.make_hparams(K, 0.1, 0.9, 0, 2)
+    w, mom, wl, pre, wdv = fake_ptrs(K)
+    host, slices, grads = 0x7f0000000000, 0x50000000, [0x60000000, 0x61000000]
+    with_pre = B.Context([n], hp, w, mom, wl, pre, wdv)
+    with pytest.raises(B.SsdError) as e:                       # pre_weight already lives on the device
+        with_pre.ssd_set_host_pre_weight(host, slices, 2)
+    assert e.value.status == B.SSD_ERR_STATE
+    ctx = B.Context([n], hp, w, mom, wl, None, wdv)            # created without pre_weight buffers
+    for call in (lambda: ctx.ssd_step(grads), lambda: ctx.ssd_step_tensors(grads, 0, 1),
+                 lambda: ctx.ssd_worker_glu_update(0, grads[0], 0), lambda: ctx.ssd_worker_local_step(0, grads[0]),
+                 lambda: ctx.ssd_step_host(grads, grads)):
+        with pytest.raises(B.SsdError) as e:
+            call()
+        assert e.value.status == B.SSD_ERR_STATE
+    for args, status in (((host, slices, 0), B.SSD_ERR_ARG), ((host, slices, 9), B.SSD_ERR_ARG),
+                         ((None, slices, 2), B.SSD_ERR_ARG), ((host, None, 2), B.SSD_ERR_ARG),
+                         ((host + 4, slices, 2), B.SSD_ERR_ALIGN), ((host, slices + 8, 2), B.SSD_ERR_ALIGN),
+                         ((host, wl[0] - 64, 1), B.SSD_ERR_ARG)):          # slices reaching into the state
+        with pytest.raises(B.SsdError) as e:
+            ctx.ssd_set_host_pre_weight(*args)
+        assert e.value.status == status
+    for bad in (1000, 1 << 31, -1024):
+        with pytest.raises(B.SsdError):
+            ctx.ssd_set_host_chunk(bad)
+    ctx.ssd_set_host_chunk(2048)
+    ctx.ssd_set_host_pre_weight(host, slices, 2)
+    with pytest.raises(B.SsdError) as e:                       # the slices were sized for the chunk
+        ctx.ssd_set_host_chunk(4096)
+    assert e.value.status == B.SSD_ERR_STATE
+    with pytest.raises(B.SsdError) as e:                       # still no device pre_weight for the fused step
+        ctx.ssd_step(grads)
+    assert e.value.status == B.SSD_ERR_STATE
+    ctx.ssd_set_host_pre_weight(None, None, 0)
+    ctx.ssd_set_host_chunk(0)
+    # without a delay stage, or with the plain-SGD updater, there is no pre_weight to place
+    with pytest.raises(B.SsdError) as e:
+        B.Context([n], B.make_hparams(K, 0.1, 0.9, 0, 0), w, mom, wl, None, wdv).ssd_set_host_pre_weight(host, slices, 2)
+    assert e.value.status == B.SSD_ERR_STATE
+    assert ctx.ssd_kernel_launches() == 0
+
+
+def test_guard_words_catch_a_store_outside_an_arena():
+    import torch
+    from paper_2012_05396_b200.state import ArenaSlab, GUARD_WORD
+    slab = ArenaSlab(3, 1001, torch.float32, "cpu")
+    assert all(a.numel() == 1001 and a.data_ptr() % 16 == 0 for a in slab.arenas)
+    for a in slab.arenas:
+        a.fill_(1.0)                                           # writes inside the arenas leave the guards alone
+    assert slab.guards_intact()
+    words = slab.raw.view(torch.int32)
+    base = slab.raw.data_ptr()
+    first_past = (slab.arenas[1].data_ptr() - base) // 4 + 1001
+    words[first_past] = 0                                      # one element past the end of arena 1
+    assert slab.damaged_gaps() == [2]
+    words[first_past] = GUARD_WORD
+    words[(slab.arenas[0].data_ptr() - base) // 4 - 1] = 7     # one element before arena 0
+    words[-1] = 7                                              # the last word of the allocation
+    assert slab.damaged_gaps() == [0, 3]

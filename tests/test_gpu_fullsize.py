@@ -90,13 +90,87 @@ def test_config_resnet50_K8_per_tensor_hyper_parameters_sampled():
     run_sampled("resnet50", 8, 8, 4, 24, 1e-3, 0.1, 0.9, per_tensor=True)
 
 
-def test_config_vgg16_K16_sampled():
-    # VGG-16 layout (138M parameters), K=16, sigma 1e-3, lr 0.01, m 0.9, W=4, k=4, 20 iterations:
-    # the workload and launch shape bench.py times
-    need = (2 + 4 * 16) * 138357544 * 4 * 1.1
+class ThreadedOracle:
+    """The CPU oracle, as it stands, run by several host threads on disjoint element ranges of one
+    slice (the update is elementwise in the parameter index; the C calls release the interpreter lock)."""
+
+    def __init__(self, ohp, w0_slice, threads):
+        from concurrent.futures import ThreadPoolExecutor
+        n = w0_slice.shape[0]
+        self.bounds = [n * t // threads for t in range(threads + 1)]
+        self.parts = [oracle.State(ohp, w0_slice[lo:hi]) for lo, hi in zip(self.bounds, self.bounds[1:])]
+        self.pool = ThreadPoolExecutor(threads)
+
+    def step(self, grads):
+        def one(t):
+            lo, hi = self.bounds[t], self.bounds[t + 1]
+            return self.parts[t].step([g[lo:hi] for g in grads])
+        return list(self.pool.map(one, range(len(self.parts))))[0]
+
+    def buffer(self, name, worker=None):
+        pick = (lambda st: getattr(st, name)) if worker is None else (lambda st: getattr(st, name)[worker])
+        return np.concatenate([pick(st) for st in self.parts])
+
+    def close(self):
+        self.pool.shutdown()
+
+
+def test_config_vgg16_K16_every_element():
+    # VGG-16 layout (138M parameters), K=16, sigma 1e-3, lr 0.01, m 0.9, W=4, k=4, 20 iterations: the
+    # workload and launch shape bench.py times.  The GPU runs the whole schedule at full size; then the
+    # oracle follows EVERY element through the same schedule, one slice of 2^24 elements at a time
+    # (gradients regenerated for the slice from the counter-based stream, host memory bounded), and all
+    # 2 + 3K buffers of the slice are compared bit for bit.
+    import os
+    K, W, k, iters, sigma = 16, 4, 4, 20, 1e-3
+    lay = synth.get_layout("vgg16")
+    N = lay.padded_numel
+    need = ((2 + 4 * K) * N * 4 + (8 << 30))
     if torch.cuda.mem_get_info()[0] < need:
         pytest.skip("not enough free device memory for the VGG-16 K=16 state")
-    run_sampled("vgg16", 16, 4, 4, 20, 1e-3, 0.01, 0.9)
+    ohp, chp = make_hp(K, 0.01, 0.9, W, k)
+    w0 = synth.init_weights(lay, device="cuda")
+    dev = DeviceState(lay.numels, chp, w0)
+    mask = synth.valid_mask(lay, "cuda") if N != lay.numel else None
+    for n in range(iters):
+        grads = [synth.gradient(lay, n, i, sigma, device="cuda", mask=mask) for i in range(K)]
+        dev.ctx.ssd_step(grads)
+        del grads
+    torch.cuda.synchronize()
+    assert dev.ctx.ssd_kernel_launches() == iters and dev.guards_intact()
+
+    threads = max(1, len(os.sched_getaffinity(0)))
+    slice_elems = 1 << 24
+    keys = [[synth.stream_key(synth.SEED, synth.STREAM_GRAD, n, i) for i in range(K)] for n in range(iters)]
+    stage_buf = torch.empty((K, slice_elems), dtype=torch.float32).pin_memory()
+    compared = 0
+    for lo in range(0, N, slice_elems):
+        hi = min(N, lo + slice_elems)
+        idx = torch.arange(lo, hi, dtype=torch.int64, device="cuda")
+        ref = ThreadedOracle(ohp, w0[lo:hi].cpu().numpy(), threads)
+        host = stage_buf[:, :hi - lo]
+        for n in range(iters):
+            for i in range(K):
+                g = synth.normal_at(keys[n][i], idx, sigma)
+                if mask is not None:
+                    g = g * mask[lo:hi]
+                host[i].copy_(g, non_blocking=True)
+            torch.cuda.synchronize()
+            ref.step([host[i].numpy() for i in range(K)])
+        tag = f"vgg16 K=16 elements [{lo}, {hi})"
+        assert_same(dev.w[lo:hi], ref.buffer("w"), tag + " w")
+        assert_same(dev.mom[lo:hi], ref.buffer("mom"), tag + " mom")
+        for i in range(K):
+            for name in ("w_loc", "pre", "w_dev"):
+                assert_same(getattr(dev, name)[i][lo:hi], ref.buffer(name, i), f"{tag} {name}[{i}]")
+        assert (ref.parts[0].iter, ref.parts[0].loc_update) == dev.ctx.ssd_get_counters()[:2]
+        ref.close()
+        compared += hi - lo
+    assert compared == N
+    # the regenerated slices really are the full-size run's gradients
+    g = synth.gradient(lay, 3, 5, sigma, device="cuda", mask=mask)
+    idx = torch.arange(N - 4096, N, dtype=torch.int64, device="cuda")
+    assert torch.equal(g[N - 4096:], synth.normal_at(keys[3][5], idx, sigma) * (1 if mask is None else mask[N - 4096:]))
 
 
 def sweep_buffer(stream, n, worker, device, idx=None):

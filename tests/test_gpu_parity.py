@@ -247,7 +247,8 @@ def test_every_kernel_shape_and_alignment_gives_the_same_bits(bf16):
         assert view.data_ptr() % 32 == 16 and view.data_ptr() % 16 == 0
         return view
 
-    for vw, batch in [(0, 0), (8, 1), (8, 2), (8, 4), (8, 8), (4, 1), (4, 2), (4, 4), (4, 8)]:
+    for vw, batch in [(0, 0), (16, 1), (16, 2), (16, 4), (16, 8), (8, 1), (8, 2), (8, 4), (8, 8), (4, 1), (4, 2),
+                      (4, 4), (4, 8)]:
         for mode in ("fused", "split"):
             dev = DeviceState(lay.numels, chp, w0)
             dev.ctx.ssd_set_kernel_shape(vw, batch)
@@ -265,6 +266,7 @@ def test_every_kernel_shape_and_alignment_gives_the_same_bits(bf16):
     dev = DeviceState(lay.numels, chp, w0)
     state = DeviceState.__new__(DeviceState)
     state.numels, state.n, state.K, state.device = dev.numels, dev.n, K, dev.device
+    state.slabs = []
     state.w, state.mom = offset_copy(dev.w, 4), offset_copy(dev.mom, 4)
     state.w_loc = [offset_copy(t, 4) for t in dev.w_loc]
     state.pre = [offset_copy(t, 4) for t in dev.pre]
@@ -297,7 +299,7 @@ def test_per_tensor_scales_and_lr_schedule(mode, bf16):
     ohp.set_tensor_scales(tensor_ends(lay), lr_mult, wd_mult)
     w0 = synth.init_weights(lay)
     ref = oracle.State(ohp, w0.numpy())
-    for vw in (0, 4):
+    for vw in (0, 4, 16):
         dev = DeviceState(lay.numels, chp, w0)
         dev.ctx.ssd_set_kernel_shape(vw, 0)
         table = torch.empty(dev.ctx.ssd_tensor_table_bytes(), dtype=torch.uint8, device="cuda")
@@ -348,7 +350,7 @@ def test_shared_pre_weight_gives_the_same_results(bf16):
     lay = synth.get_layout("resnet20")
     ohp, chp = make_hp(K, 0.1, 0.9, W, k, wd=1e-3, bf16=bf16)
     w0 = synth.init_weights(lay)
-    for vw, batch in ((0, 0), (4, 4), (8, 2)):
+    for vw, batch in ((0, 0), (4, 4), (8, 2), (16, 1)):
         dev = DeviceState(lay.numels, chp, w0, shared_pre=True)
         assert len({t.data_ptr() for t in dev.pre}) == 1
         dev.ctx.ssd_set_kernel_shape(vw, batch)
@@ -527,7 +529,7 @@ def test_random_combinations_of_every_option():
         local_sgd = bool(rng.integers(4) == 0)
         shared = bool(rng.integers(2)) and K > 1 and k > 0
         issue = str(rng.choice(["step", "layers"] if shared else ["step", "layers", "split"]))
-        vw, batch = int(rng.choice([0, 4, 8])), int(rng.choice([0, 1, 2, 4, 8]))
+        vw, batch = int(rng.choice([0, 4, 8, 16])), int(rng.choice([0, 1, 2, 4, 8]))
         iters = W + 2 * max(k, 1) + 2
         tag = f"case {case}: numels={numels} K={K} W={W} k={k} bf16={bf16} pt={per_tensor} sgd={local_sgd} " \
               f"shared={shared} issue={issue} shape=({vw},{batch})"

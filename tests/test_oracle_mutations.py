@@ -48,6 +48,10 @@ MUTATIONS = [
     ("tensor lookup off by one", "pos >= hp->tensor_end[t]", "pos > hp->tensor_end[t]"),
     ("local lr ignores the tensor's multiplier", "float lr_loc_t = hp->lr_loc * hp->lr_mult[t];", "float lr_loc_t = hp->lr_loc;"),
     ("decay multiplier taken from lr_mult", "float wd_t = hp->wd * hp->wd_mult[t];", "float wd_t = hp->wd * hp->lr_mult[t];"),
+    ("server flushes subnormal momenta to zero", "mom[j] = keep - step;",
+     "mom[j] = keep - step; if (mom[j] > -1.17549435e-38f && mom[j] < 1.17549435e-38f) mom[j] = 0;"),
+    ("GLU flushes a subnormal grad_sync to zero", "real grad_sync = diff * c;",
+     "real grad_sync = diff * c; if (grad_sync > -1.17549435e-38f && grad_sync < 1.17549435e-38f) grad_sync = 0;"),
     ("per-tensor scale from the global lr", "s.c = sync_scale_for(lr_t, hp->m, hp->k);", "s.c = sync_scale_for(hp->lr, hp->m, hp->k);"),
 ]
 
@@ -100,6 +104,7 @@ def traces_pass(lib):
         try:
             test_oracle_pins.test_local_sgd_updater_is_eq5_and_never_touches_pre_weight()
             test_oracle_pins.test_local_sgd_equals_glu_with_alpha_one_beta_zero()
+            test_oracle_pins.test_subnormals_are_kept_not_flushed_exact_dyadic_case()
         except AssertionError:
             return False
         return True

@@ -616,3 +616,160 @@ def test_brute_force_random_hyper_parameters():
                 np.testing.assert_array_equal(st.pre[i], np.array(pre[i], f32))
             if w_dev[i][0] is not None:
                 np.testing.assert_array_equal(st.w_dev[i], np.array(w_dev[i], f32))
+
+
+# ---------------------------------------------------------------------------
+# the ends of the binary32 range: gradual underflow (no flush to zero), signed zeros,
+# overflow to infinity.  The paper is silent on rounding; the reading is IEEE 754
+# binary32, round to nearest even, every operation rounded on its own, subnormals kept.
+# The expected values are exact rational arithmetic with that rounding written out.
+# ---------------------------------------------------------------------------
+
+from fractions import Fraction
+
+
+def rn32(x: Fraction) -> float:
+    """Round a rational to binary32, nearest even, with gradual underflow; overflow gives inf."""
+    if x == 0:
+        return 0.0
+    sign = -1 if x < 0 else 1
+    a = abs(x)
+    e = -126                                   # exponent of the binade that holds a, subnormals share -126
+    while a >= Fraction(2) ** (e + 1):
+        e += 1
+    quantum = Fraction(2) ** (e - 23)
+    q = a / quantum
+    n = q.numerator // q.denominator
+    rem = q - n
+    if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and n % 2 == 1):
+        n += 1
+    r = n * quantum
+    if r >= Fraction(2) ** 128:
+        return sign * float("inf")
+    return sign * float(r)                     # exact: r has at most 24 significant bits
+
+
+def _finite(*xs):
+    return all(np.isfinite(x) for x in xs)
+
+
+def xmul(a, b) -> float:
+    """binary32 product of two binary32 values (Python floats), exactly rounded."""
+    a, b = float(a), float(b)
+    if not _finite(a, b):
+        with np.errstate(all="ignore"):
+            return float(np.float64(a) * np.float64(b))         # inf and NaN rules do not depend on the width
+    r = rn32(Fraction(a) * Fraction(b))
+    negative = np.signbit(a) != np.signbit(b)
+    return -abs(r) if negative else abs(r)                       # also fixes the sign of a zero product
+
+
+def xadd(a, b) -> float:
+    a, b = float(a), float(b)
+    if not _finite(a, b):
+        with np.errstate(all="ignore"):
+            return float(np.float64(a) + np.float64(b))
+    exact = Fraction(a) + Fraction(b)
+    if exact == 0:                                               # x + (-x) = +0; (-0) + (-0) = -0
+        return -0.0 if (a == 0 and b == 0 and np.signbit(a) and np.signbit(b)) else 0.0
+    return rn32(exact)
+
+
+def xsub(a, b) -> float:
+    return xadd(a, -float(b))
+
+
+def exact_server(g, w, mom, lr, m, wd, rescale):
+    s = float(g[0])
+    for gi in g[1:]:
+        s = xadd(s, gi)
+    grad = xmul(s, rescale)
+    full = xadd(grad, xmul(wd, w))
+    step = xmul(lr, full)
+    keep = xmul(m, mom)
+    mom2 = xsub(keep, step)
+    return xadd(w, mom2), mom2
+
+
+def exact_glu(g, wl, pre, lr_loc, alpha, beta, wd, c):
+    gs = xmul(xsub(pre, wl), c)
+    mix = xadd(xmul(alpha, g), xmul(wd, wl))
+    mix = xadd(mix, xmul(beta, gs))
+    return xsub(wl, xmul(lr_loc, mix))
+
+
+def test_rounding_helper_against_known_values():
+    tiny = 2.0 ** -149
+    assert rn32(Fraction(1, 3)) == float(f32(1.0) / f32(3.0))
+    assert rn32(Fraction(2) ** -150) == 0.0                       # tie between 0 and the smallest subnormal: even
+    assert rn32(3 * Fraction(2) ** -150) == 2 * tiny              # tie between 1 and 2 quanta: even
+    assert rn32(Fraction(2) ** -150 + Fraction(2) ** -200) == tiny
+    assert rn32(Fraction(2) ** 128 - Fraction(2) ** 103) == float("inf")     # half a quantum above the largest
+    assert rn32(Fraction(2) ** 128 - Fraction(2) ** 103 - 1) == float(np.finfo(f32).max)
+    assert rn32(Fraction(16777217)) == 16777216.0 and rn32(Fraction(16777219)) == 16777220.0
+
+
+def test_subnormals_are_kept_not_flushed_exact_dyadic_case():
+    # every operand and every intermediate is a multiple of 2^-149 below 2^-126 or an exact dyadic
+    # product, so nothing is rounded: the results are the exact values of the formulas of
+    # Section 3.2.1 and 3.3 and are subnormal.  A flush to zero anywhere gives other numbers.
+    u = 2.0 ** -149
+    lr, m, wd, K = 0.5, 0.5, 0.25, 2
+    g = [f32(24 * u), f32(40 * u)]                               # sum 64u, averaged 32u
+    w, mom = f32(1024 * u), f32(-96 * u)                         # wd*w = 256u, lr*(32u+256u) = 144u, m*mom = -48u
+    hp = Hyper(K=K, lr=lr, m=m, W=0, k=2, wd=wd, lr_loc=2.0, alpha=2.0, beta=0.5)
+    wa, ma = np.array([w], f32), np.array([mom], f32)
+    oracle.server_update(hp, [np.array([x], f32) for x in g], wa, ma)
+    assert ma[0] == f32(-192 * u) and wa[0] == f32(832 * u)
+    assert (float(wa[0]), float(ma[0])) == exact_server(g, w, mom, lr, m, wd, 1.0 / K)
+    assert 0 < abs(float(ma[0])) < 2.0 ** -126                   # subnormal results, not zero
+    # GLU: c = (1-m)/(lr*k) = 0.5; (pre - w') = 64u, grad_sync = 32u; alpha*g = 48u, wd*w' = 128u,
+    # mix = 176u + beta*32u = 192u; w' - lr_loc*192u = 512u - 384u = 128u
+    assert oracle.sync_scale(hp) == 0.5
+    wl, pre, dev = np.array([512 * u], f32), np.array([576 * u], f32), np.zeros(1, f32)
+    oracle.glu_update(hp, np.array([24 * u], f32), wl, pre, dev, None, 0)
+    assert wl[0] == f32(128 * u) and pre[0] == f32(576 * u)
+    assert float(wl[0]) == exact_glu(f32(24 * u), f32(512 * u), f32(576 * u), 2.0, 2.0, 0.5, wd, 0.5)
+
+
+def test_range_ends_against_exact_rational_arithmetic():
+    # operands drawn from both ends of the binary32 range, with rounding inside the subnormal
+    # range, sums that cancel to +0, and overflow to infinity; expected values from exact
+    # rational arithmetic rounded to nearest even operation by operation
+    u = 2.0 ** -149
+    big = float(np.finfo(f32).max)
+    pool = [0.0, u, 3 * u, 5 * u, 2.0 ** -127, 2.0 ** -126, 1.5 * 2.0 ** -126, 7 * 2.0 ** -130, 1e-38, 1e-40,
+            1.0, 0.1, big, big / 2, 2.0 ** 127, 1e38]
+    rng = np.random.default_rng(12)
+    lr, m, wd, lr_loc, alpha, beta = 0.1, 0.9, 0.01, 0.4, 2.0, 0.5
+    n_sub = n_inf = n_zero = 0
+    for K in (1, 2, 3):
+        hp = Hyper(K=K, lr=lr, m=m, W=0, k=4, wd=wd, lr_loc=lr_loc, alpha=alpha, beta=beta)
+        c = oracle.sync_scale(hp)
+        for trial in range(400):
+            draw = lambda: f32(rng.choice(pool) * rng.choice([-1.0, 1.0]))
+            g = [draw() for _ in range(K)]
+            w, mom, wl, pre = draw(), draw(), draw(), draw()
+            if trial % 5 == 0:
+                pre = wl                                         # grad_sync exactly +0
+            exp_w, exp_mom = exact_server(g, w, mom, f32(lr), f32(m), f32(wd), hp.rescale)
+            wa, ma = np.array([w], f32), np.array([mom], f32)
+            with np.errstate(all="ignore"):
+                oracle.server_update(hp, [np.array([x], f32) for x in g], wa, ma)
+            if np.isnan(exp_mom) or np.isnan(exp_w):             # inf - inf: only "is a NaN" is defined
+                assert np.isnan(ma[0]) or np.isnan(wa[0])
+            else:
+                assert (float(wa[0]), float(ma[0])) == (exp_w, exp_mom), (K, trial, g, w, mom)
+                assert np.signbit(wa[0]) == np.signbit(f32(exp_w))           # the sign of a zero counts too
+            exp_wl = exact_glu(g[0], wl, pre, f32(lr_loc), f32(alpha), f32(beta), f32(wd), f32(c))
+            la, pa, da = np.array([wl], f32), np.array([pre], f32), np.zeros(1, f32)
+            oracle.glu_update(hp, np.array([g[0]], f32), la, pa, da, None, 0)
+            if np.isnan(exp_wl):
+                assert np.isnan(la[0])
+            else:
+                assert float(la[0]) == exp_wl and np.signbit(la[0]) == np.signbit(f32(exp_wl)), (K, trial)
+            for v in (exp_mom, exp_w, exp_wl):
+                n_sub += 0 < abs(v) < 2.0 ** -126
+                n_inf += np.isinf(v)
+                n_zero += v == 0
+    assert n_sub > 200 and n_inf > 50 and n_zero > 10            # the draw really reaches all three regimes
