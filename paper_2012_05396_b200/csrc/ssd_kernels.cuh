@@ -52,6 +52,7 @@ struct SyncParams {
     float *w, *mom;
     int64_t n;
     int K, flags;
+    int per_batch;                 // workers per batch of loads: K split evenly over ceil(K / B) batches
     Scalars s;
     TensorTable tt;
 };
@@ -74,6 +75,7 @@ struct StepParams {
     float *w, *mom;
     int64_t n;
     int K, flags;
+    int per_batch;                 // workers per batch of loads: K split evenly over ceil(K / B) batches
     int shared_pre;                // 1: pre[0] is the one pre_weight of all workers
     Scalars s;
     TensorTable tt;
@@ -303,14 +305,16 @@ __device__ __forceinline__ void sync_at(const SyncParams &p, int64_t e)
     Vec<VW> w = ld_f32<VW>(p.w, e);
     Vec<VW> mom = ld_f32<VW>(p.mom, e);
     Vec<VW> sum;
-    for (int i0 = 0; i0 < p.K; i0 += B) {
+    // batches of at most B workers, all of (nearly) the same size: 9 workers with B = 8 go as 5 + 4
+    const int per = p.per_batch;
+    for (int i0 = 0; i0 < p.K; i0 += per) {
         Grad<GT, VW> g[B];
 #pragma unroll
         for (int b = 0; b < B; ++b)
-            if (i0 + b < p.K) g[b] = ld_grad<GT, VW>(p.g[i0 + b], e);
+            if (b < per && i0 + b < p.K) g[b] = ld_grad<GT, VW>(p.g[i0 + b], e);
 #pragma unroll
         for (int b = 0; b < B; ++b) {
-            if (i0 + b < p.K) {
+            if (b < per && i0 + b < p.K) {
 #pragma unroll
                 for (int l = 0; l < VW; ++l)
                     sum.v[l] = (i0 + b == 0) ? g[b].get(l) : __fadd_rn(sum.v[l], g[b].get(l));
@@ -365,12 +369,13 @@ __device__ __forceinline__ void step_at(const StepParams &p, int64_t e)
     Vec<VW> pre_shared;
     if (shared && !first && !sgd) pre_shared = ld_f32<VW>(p.pre[0], e);
     GroupScalars<PT, VW> sc(p.s, p.tt, e);
-    for (int i0 = 0; i0 < p.K; i0 += B) {
+    const int per = p.per_batch;
+    for (int i0 = 0; i0 < p.K; i0 += per) {
         Grad<GT, VW> g[B];
         Vec<VW> wl[B], pr[B];
 #pragma unroll
         for (int b = 0; b < B; ++b) {
-            if (i0 + b < p.K) {
+            if (b < per && i0 + b < p.K) {
                 g[b] = ld_grad<GT, VW>(p.g[i0 + b], e);
                 wl[b] = ld_f32<VW>(p.w_loc[i0 + b], e);
                 if (!first && !shared && !sgd) pr[b] = ld_f32<VW>(p.pre[i0 + b], e);
@@ -378,7 +383,7 @@ __device__ __forceinline__ void step_at(const StepParams &p, int64_t e)
         }
 #pragma unroll
         for (int b = 0; b < B; ++b) {
-            if (i0 + b < p.K) {
+            if (b < per && i0 + b < p.K) {
                 const int i = i0 + b;
                 Vec<VW> r;
 #pragma unroll

@@ -228,32 +228,60 @@ Shape sync_shape(const ssd_ctx *c, int max_vw)
 {
     const int K = c->hp.K;
     Shape sh;
-    if (c->hp.grad_dtype == SSD_BF16)
-        sh = K >= 4 ? Shape{8, 4, 128, 6} : Shape{8, 1, 128, K == 1 ? 4 : 6};
-    else
-        sh = K >= 4 ? Shape{8, 4, 128, 5} : Shape{8, 1, 128, 6};
+    // (the batch is an upper bound: the K workers go in ceil(K / batch) batches of equal size)
+    if (c->hp.grad_dtype == SSD_BF16) {
+        // bfloat16 gradients: vectors of 16 fetch them with 256-bit loads like the float32 state
+        // (with vectors of 8 a warp asks for 512 contiguous bytes of a gradient stream at a time and
+        // the kernel stays 7 % below its float32 twin)
+        if (K >= 16) sh = Shape{16, 8, 128, 3};
+        else if (K >= 7) sh = Shape{16, 8, 128, 4};
+        else if (K >= 5) sh = Shape{16, 8, 128, 3};
+        else if (K == 4) sh = Shape{16, 4, 128, 3};
+        else if (K == 3) sh = Shape{8, 4, 128, 6};
+        else if (K == 2) sh = Shape{16, 2, 128, 4};
+        else sh = Shape{16, 1, 128, 4};
+        if (max_vw < 16) sh = K >= 3 ? Shape{8, 4, 128, 6} : Shape{8, 1, 128, K == 1 ? 4 : 6};
+    } else {
+        if (K >= 8 || K == 4) sh = Shape{8, 4, 128, 5};
+        else if (K >= 5) sh = Shape{8, 8, 128, 4};
+        else if (K == 3) sh = Shape{16, 4, 128, 3};
+        else if (K == 2) sh = Shape{16, 2, 128, 3};
+        else sh = Shape{8, 1, 128, 6};
+        if (max_vw < 16 && K < 4) sh = K == 3 ? Shape{8, 4, 128, 5} : Shape{8, 1, 128, 6};
+    }
     return finish_shape(c, sh, max_vw, 8);
 }
 
 Shape step_shape(const ssd_ctx *c, int flags, bool shared_pre, int max_vw, int64_t count)
 {
     // Iterations that add K stores per element (pull; refresh or first call with one pre_weight
-    // per worker) are write-heavy: 512 threads per SM.  The others: 640 threads per SM.
+    // per worker) are write-heavy: 512 threads per SM with vectors of 8.  The others: 640 threads
+    // per SM.  Vectors of 16 (384 threads per SM) win where gradients are bfloat16 and the iteration
+    // is write-heavy, and on plain iterations with one or two workers.
+    const int K = c->hp.K;
+    const bool bf16 = c->hp.grad_dtype == SSD_BF16;
     const bool sgd = c->hp.local_updater == SSD_LOCAL_SGD;
     const bool k_extra_stores = (flags & kPull) || (!shared_pre && !sgd && (flags & (kRefresh | kFirst)));
     Shape sh = k_extra_stores ? Shape{8, 1, 128, 4} : Shape{8, 1, 128, 5};
+    if (max_vw >= 16) {
+        if (k_extra_stores && bf16) sh = Shape{16, 1, 128, 3};
+        if (!k_extra_stores && (K == 1 || (K == 2 && !bf16))) sh = Shape{16, 1, 128, 3};
+    }
     // A step whose whole traffic fits in L2 (ResNet-20/56 sized arenas) is bound by latency, not by
     // DRAM: smaller vectors spread it over more threads, and two workers' loads per thread halve the
     // number of dependent round trips.
-    const int64_t sg = c->hp.grad_dtype == SSD_BF16 ? 2 : 4;
-    if (count * (c->hp.K * (sg + 12) + 16) < kL2ResidentBytes) sh = Shape{4, 2, 64, 0};
+    const int64_t sg = bf16 ? 2 : 4;
+    if (count * (K * (sg + 12) + 16) < kL2ResidentBytes) sh = Shape{4, 2, 64, 0};
     sh = finish_shape(c, sh, max_vw, 4);
     // batches that would spill registers under the kernels' thread bounds
     if (sh.vw >= 8 && sh.batch > 2) sh.batch = 2;
     return sh;
 }
 
-Shape glu_shape(const ssd_ctx *c, int max_vw) { return finish_shape(c, Shape{8, 1, 256, 0}, max_vw, 1); }
+Shape glu_shape(const ssd_ctx *c, int max_vw)
+{
+    return finish_shape(c, max_vw >= 16 ? Shape{16, 1, 128, 0} : Shape{8, 1, 256, 0}, max_vw, 1);
+}
 
 size_t table_end_bytes(const ssd_ctx *c) { return (c->offsets.size() * sizeof(int64_t) + 15) / 16 * 16; }
 size_t table_bytes(const ssd_ctx *c) { return table_end_bytes(c) + c->offsets.size() * sizeof(float4); }
@@ -339,9 +367,18 @@ ssd_status check_grads(const ssd_ctx *c, const void *const *grads)
     return SSD_OK;
 }
 
-template <int GT, int VW, bool PT>
-ssd_status launch_sync_b(ssd_ctx *c, const SyncParams &p, const Shape &sh, cudaStream_t stream)
+// K workers in ceil(K / batch) batches of equal size (the last one may be smaller by less than a batch).
+int even_batch(int K, int batch)
 {
+    const int batches = (K + batch - 1) / batch;
+    return (K + batches - 1) / batches;
+}
+
+template <int GT, int VW, bool PT>
+ssd_status launch_sync_b(ssd_ctx *c, SyncParams &p, const Shape &sh, cudaStream_t stream)
+{
+    const int compiled = sh.batch >= 8 ? ((VW == 16 && GT == kF32) ? 4 : 8) : sh.batch >= 4 ? 4 : sh.batch >= 2 ? 2 : 1;
+    p.per_batch = even_batch(p.K, compiled);
     switch (sh.batch) {
     case 1: return launch(c, sync_kernel<GT, VW, 1, PT>, p, p.n, sh, stream);
     case 2: return launch(c, sync_kernel<GT, VW, 2, PT>, p, p.n, sh, stream);
@@ -353,7 +390,7 @@ ssd_status launch_sync_b(ssd_ctx *c, const SyncParams &p, const Shape &sh, cudaS
 }
 
 template <bool PT>
-ssd_status launch_sync_t(ssd_ctx *c, const SyncParams &p, const Shape &sh, cudaStream_t stream)
+ssd_status launch_sync_t(ssd_ctx *c, SyncParams &p, const Shape &sh, cudaStream_t stream)
 {
     const bool bf16 = c->hp.grad_dtype == SSD_BF16;
     if (sh.vw == 16)
@@ -423,8 +460,9 @@ ssd_status launch_glu(ssd_ctx *c, int worker, const void *grad, int flags, cudaS
 }
 
 template <int GT, int VW, bool PT>
-ssd_status launch_step_b(ssd_ctx *c, const StepParams &p, const Shape &sh, cudaStream_t stream)
+ssd_status launch_step_b(ssd_ctx *c, StepParams &p, const Shape &sh, cudaStream_t stream)
 {
+    p.per_batch = even_batch(p.K, sh.batch == 1 ? 1 : (sh.batch == 2 || VW >= 8) ? 2 : 4);
     // step_shape keeps the batch at 2 or below for vectors of 8 and more (4 would spill)
     if (sh.batch == 1) return launch(c, step_kernel<GT, VW, 1, PT>, p, p.n, sh, stream);
     if constexpr (VW == 4)
@@ -433,7 +471,7 @@ ssd_status launch_step_b(ssd_ctx *c, const StepParams &p, const Shape &sh, cudaS
 }
 
 template <bool PT>
-ssd_status launch_step_t(ssd_ctx *c, const StepParams &p, const Shape &sh, cudaStream_t stream)
+ssd_status launch_step_t(ssd_ctx *c, StepParams &p, const Shape &sh, cudaStream_t stream)
 {
     const bool bf16 = c->hp.grad_dtype == SSD_BF16;
     if (sh.vw == 16)

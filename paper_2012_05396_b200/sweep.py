@@ -30,6 +30,18 @@ from .state import DeviceState, alloc_arenas
 L2_BYTES = 126e6
 
 
+def measured_peak() -> float:
+    """The HBM copy rate measured on this machine (MEASURED_PEAKS.json at the repository root), else the
+    earlier measurement of 6650 GB/s."""
+    import os
+    path = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"])
+    except Exception:
+        return 6650.0
+
+
 def time_launches(fn, reps: int, warmup: int = 3):
     stream = torch.cuda.current_stream()
     for _ in range(warmup):
@@ -155,16 +167,18 @@ def point(log2n: int, K: int, dtype: str, kernels, reps: int, peak: float, threa
                 sets.append((st, grads))
             stream = torch.cuda.current_stream()
             per_flag = {}
-            for r in range(R * (4 + max(reps, 8))):                  # every set goes through the same schedule
+            total = R * (4 + max(reps, 8))                           # every set goes through the same schedule
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(total + 1)]
+            flags_of = []
+            ev[0].record(stream)
+            for r in range(total):                                   # enqueued back to back, as a training loop does
                 st, grads = sets[r % R]
-                flags = st.ctx.ssd_get_counters()[3]
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e0.record(stream)
+                flags_of.append(st.ctx.ssd_get_counters()[3])
                 st.ctx.ssd_step(grads)
-                e1.record(stream)
-                torch.cuda.synchronize()
-                if r >= 4 * R:
-                    per_flag.setdefault(flags, []).append(e0.elapsed_time(e1))
+                ev[r + 1].record(stream)
+            torch.cuda.synchronize()
+            for r in range(4 * R, total):
+                per_flag.setdefault(flags_of[r], []).append(ev[r].elapsed_time(ev[r + 1]))
             for flags, ms in sorted(per_flag.items()):
                 b = K * (sg + 12) + 16 + (4 * K if flags & 2 else 0) + (4 * K if flags & 4 else 0)
                 name = "step" + ("+refresh" if flags & 2 else "") + ("+pull" if flags & 4 else "")
@@ -183,10 +197,12 @@ def main():
     ap.add_argument("--dtype", nargs="+", default=["f32", "bf16"], choices=["f32", "bf16"])
     ap.add_argument("--kernels", nargs="+", default=["sync", "glu", "step"], choices=["sync", "glu", "step"])
     ap.add_argument("--reps", type=int, default=20)
-    ap.add_argument("--peak", type=float, default=6547.5, help="measured HBM copy rate in GB/s")
+    ap.add_argument("--peak", type=float, default=0.0,
+                    help="HBM copy rate in GB/s for the 'of measured' column (0 = read MEASURED_PEAKS.json, "
+                         "else the pool's earlier figure of 6650)")
     ap.add_argument("--threads", type=int, default=0)
     ap.add_argument("--blocks-per-sm", type=int, default=0)
-    ap.add_argument("--vector-elems", type=int, default=0, choices=[0, 4, 8])
+    ap.add_argument("--vector-elems", type=int, default=0, choices=[0, 4, 8, 16])
     ap.add_argument("--batch", type=int, default=0, choices=[0, 1, 2, 4, 8])
     ap.add_argument("--staging", type=int, default=0,
                     help="stages of the shared-memory ring for the fused step (0 = register path)")
@@ -194,6 +210,8 @@ def main():
     if not torch.cuda.is_available():
         raise SystemExit("the sweep needs a CUDA device")
     libbuild.build_library()
+    if args.peak <= 0:
+        args.peak = measured_peak()
     for log2n in args.log2n:
         for K in args.K:
             for dtype in args.dtype:
