@@ -43,11 +43,15 @@ WORKLOADS = {
 }
 DEFAULT_WORKLOAD = "vgg16_K16"
 
-# DRAM bytes per launch of step_kernel on the default workload (dram__bytes_read.sum +
-# dram__bytes_write.sum, one-pass ncu capture of this benchmark's own launches), by iteration flags
-# (0 plain, 2 refresh, 4 pull).  Valid only for the kernel sources with this digest.
-NCU_TRAFFIC = {"digest": "33b3897842d55989", "workload": "vgg16_K16",
-               "bytes_per_launch": {0: 37601010048, 2: 46437748992, 4: 46442552320}}
+# DRAM bytes per PARAMETER of one step_kernel launch (dram__bytes_read.sum + dram__bytes_write.sum
+# from an ncu capture of a small flat arena: 2^24 parameters, K = 16 float32 workers, 4.4 GB
+# resident), by iteration flags (0 plain, 2 refresh, 4 pull).  The kernel streams every byte once,
+# so its traffic grows in proportion to the parameter count and a full-size launch is this figure
+# times its parameters.  Valid only for K = 16 float32 and the kernel sources with this digest;
+# otherwise the bench line carries traffic = null.
+NCU_TRAFFIC = {"digest": "0f87fcb100c46a58", "K": 16, "grad_dtype": "f32", "captured_params": 1 << 24,
+               "bytes_per_param": {0: 269.958, 2: 332.618, 4: 332.867}}
+TARGET_TIMED_MS = 2000.0      # repeats of the timed region are added until about this much GPU time
 
 
 def kernel_digest() -> str:
@@ -100,7 +104,7 @@ class ClockSampler:
             self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.QUERY}",
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "20"],
                 stdout=self.file, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
@@ -243,14 +247,71 @@ def run_reference(args, wl_name, wl):
     print(json.dumps(line))
 
 
+def host_step_bytes(K: int, sg: int, flags: int, stage_delay: bool, host_grads: bool, host_pre: bool,
+                    read_back: bool):
+    """(host-to-device, device-to-host) bytes per parameter of one ssd_step_host call."""
+    h2d = K * sg if host_grads else 0
+    d2h = 4 if read_back else 0
+    if host_pre and stage_delay:
+        if not flags & 1:            # every GLU call but the first reads pre_weight
+            h2d += 4
+        if flags & 3:                # the first call and the refreshes write it back
+            d2h += 4
+    return h2d, d2h
+
+
+def time_regions(run_region, repeats: int, world: int, dev_name: str):
+    """Times `repeats` regions on the current stream, each bracketed by a barrier and a device
+    synchronisation on both sides; returns per region (ms over ranks' maximum, per-step ms list)."""
+    import torch.distributed as dist
+    out = []
+    for _ in range(repeats):
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        events = run_region()
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        total = events[0].elapsed_time(events[-1])
+        steps = [events[i].elapsed_time(events[i + 1]) for i in range(len(events) - 1)]
+        out.append((max_over_ranks(total, dev_name, world), steps))
+    return out
+
+
+def kernel_table(peak: float):
+    """Every update kernel on two more workloads of 25M parameters and more, measured in this process
+    with the sweep's method (CUDA events between back-to-back launches, buffer sets rotated so that
+    nothing is served from L2): the ResNet-50 layout with K = 8 float32 workers and a flat 2^26
+    tensor with K = 16 bfloat16 workers."""
+    from paper_2012_05396_b200 import sweep, synth
+    rows = []
+    cases = [("resnet50_K8_f32", synth.get_layout("resnet50").numels, 25, 8, "f32"),
+             ("flat2p26_K16_bf16", None, 26, 16, "bf16")]
+    for name, numels, log2n, K, dtype in cases:
+        for rec in sweep.point(log2n, K, dtype, ["sync", "glu", "step"], 20, peak, numels=numels):
+            if "gbs" not in rec:
+                rows.append({"workload": name, "kernel": rec["kernel"], "skipped": rec.get("skipped")})
+                continue
+            rows.append({"workload": name, "kernel": rec["kernel"], "params": rec["params"], "workers": K,
+                         "grad_dtype": dtype, "algorithmic_bytes": rec["bytes_per_launch"],
+                         "ms": rec["ms_median"], "gbs": rec["gbs"], "frac_of_measured": rec["gbs"] / peak,
+                         "frac_of_nominal_8TBs": rec["gbs"] / NOMINAL_HBM_GBS})
+    return rows
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=4)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--repeats", type=int, default=0,
+                    help="timed regions of --steps steps each (0 = at least 5, more until about 2 s of GPU time)")
     ap.add_argument("--e2e-steps", type=int, default=4)
+    ap.add_argument("--no-host-pre", action="store_true", help="skip the host-resident pre_weight legs")
+    ap.add_argument("--no-kernel-table", action="store_true", help="skip the per-kernel table")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--per-tensor", action="store_true",
                     help="per-tensor hyper-parameters: weight decay 5e-4 on conv/FC weights only")
@@ -313,110 +374,174 @@ def main():
             arenas[i].copy_(synth.gradient(lay, s, i, wl["sigma"], device=dev_name, mask=mask))
         grad_sets.append(arenas)
     stream = torch.cuda.current_stream()
+    state_bytes = st.bytes()
+    l2_note = "inputs larger than L2 (no flush needed)" if state_bytes > 4 * 126e6 \
+        else "L2-resident: not an HBM measurement"
 
-    # SSD warm-up stage + first GLU call, then the bench's own warm-up steps (all untimed).
-    for n in range(wl["W"] + 1 + max(args.warmup, 3)):
+    # SSD warm-up stage + first GLU call, then the bench's own warm-up steps (all untimed); the
+    # last of them are timed roughly to choose the number of repeats.
+    warm = max(args.warmup, 3)
+    for n in range(wl["W"] + 1):
         st.ctx.ssd_step(grad_sets[n % n_sets])
     torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for n in range(warm):
+        st.ctx.ssd_step(grad_sets[n % n_sets])
+    torch.cuda.synchronize()
+    est_region_ms = (time.perf_counter() - t0) / warm * args.steps * 1e3
+    est_region_ms = max_over_ranks(est_region_ms, dev_name, world)
+    repeats = args.repeats or int(min(50, max(5, -(-TARGET_TIMED_MS // max(est_region_ms, 1e-3)))))
 
-    flags_of = []
-    it0 = st.ctx.ssd_get_counters()[0]
-    for n in range(args.steps):
-        flags_of.append(st.ctx.ssd_schedule(it0 + n)[1])
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    flags_per_region = []
     launches0 = st.ctx.ssd_kernel_launches()
+
+    def region():
+        it0 = st.ctx.ssd_get_counters()[0]
+        flags_per_region.append([st.ctx.ssd_schedule(it0 + n)[1] for n in range(args.steps)])
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+        ev[0].record(stream)
+        for n in range(args.steps):
+            st.ctx.ssd_step(grad_sets[n % n_sets])
+            ev[n + 1].record(stream)
+        return ev
 
     sampler = ClockSampler(local)
     sampler.start()
     time.sleep(0.3)
-    if world > 1:
-        dist.barrier()
-    torch.cuda.synchronize()
     t_wall = time.perf_counter()
-    ev[0].record(stream)
-    for n in range(args.steps):
-        st.ctx.ssd_step(grad_sets[n % n_sets])
-        ev[n + 1].record(stream)
-    torch.cuda.synchronize()
+    regions = time_regions(region, repeats, world, dev_name)
     t_wall = time.perf_counter() - t_wall
-    if world > 1:
-        dist.barrier()
     clocks = sampler.stop()
     launches = st.ctx.ssd_kernel_launches() - launches0
 
-    total_ms = ev[0].elapsed_time(ev[-1])
-    per_launch_ms = [ev[n].elapsed_time(ev[n + 1]) for n in range(args.steps)]
-    total_ms = max_over_ranks(total_ms, dev_name, world)
-    bytes_per_launch = [step_bytes_per_param(K, sg, f, args.shared_pre, args.local_sgd) * N for f in flags_of]
-    value = whole_job_rate(float(sum(bytes_per_launch)), world, total_ms) / 1e9
+    def region_bytes(flags):
+        return [step_bytes_per_param(K, sg, f, args.shared_pre, args.local_sgd) * N for f in flags]
+
+    rates = [whole_job_rate(float(sum(region_bytes(f))), world, ms) / 1e9
+             for f, (ms, _) in zip(flags_per_region, regions)]
+    order = sorted(range(repeats), key=lambda r: rates[r])
+    mid = order[repeats // 2]                                     # the median region is the one reported
+    value, total_ms, per_launch_ms = rates[mid], regions[mid][0], regions[mid][1]
+    bytes_per_launch = region_bytes(flags_per_region[mid])
     peak, peak_kind = measured_peak()
-    achieved = (sum(bytes_per_launch) / len(bytes_per_launch)) / (statistics.mean(per_launch_ms) * 1e-3) / 1e9
+    # the dominant (only) kernel of the timed region: mean over every launch of every region
+    all_ms = [ms for _, steps in regions for ms in steps]
+    all_bytes = [b for f in flags_per_region for b in region_bytes(f)]
+    achieved = (sum(all_bytes) / len(all_bytes)) / (statistics.mean(all_ms) * 1e-3) / 1e9
+    by_flags = {}
+    for f, (_, steps) in zip(flags_per_region, regions):
+        for fl, ms in zip(f, steps):
+            by_flags.setdefault(fl & 6, []).append(ms)
+    names = {0: "plain", 2: "refresh", 4: "pull", 6: "refresh+pull"}
+    per_kind = {names[fl]: {"launches": len(ms), "ms_median": statistics.median(ms),
+                            "gbs": step_bytes_per_param(K, sg, fl, args.shared_pre, args.local_sgd) * N
+                            / (statistics.median(ms) * 1e-3) / 1e9}
+                for fl, ms in sorted(by_flags.items())}
     traffic = None
-    if (NCU_TRAFFIC["digest"] == kernel_digest() and NCU_TRAFFIC["workload"] == wl_name
-            and not args.shared_pre and not args.local_sgd and not args.per_tensor and not args.threads and not args.blocks_per_sm):
-        per = NCU_TRAFFIC["bytes_per_launch"]
-        if all((f & 6) in per for f in flags_of):
-            traffic = statistics.mean(per[f & 6] for f in flags_of)
+    plain_config = not (args.shared_pre or args.local_sgd or args.per_tensor or args.threads or args.blocks_per_sm)
+    if NCU_TRAFFIC["digest"] == kernel_digest() and NCU_TRAFFIC["K"] == K and plain_config:
+        per = NCU_TRAFFIC["bytes_per_param"]
+        kinds = [f & 6 for fl in flags_per_region for f in fl]
+        if all(kd in per for kd in kinds):
+            traffic = statistics.mean(per[kd] for kd in kinds) * N
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+        "warmup": warm, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "repeats": {"count": repeats, "reported": "median", "value_min": min(rates), "value_max": max(rates),
+                    "timed_ms_total": sum(ms for ms, _ in regions)},
         "params_per_s": whole_job_rate(float(N) * args.steps, world, total_ms),
         "frac_of_nominal_8TBs": value / world / NOMINAL_HBM_GBS,
-        "wall_ms_per_step": t_wall / args.steps * 1e3,
+        "wall_ms_per_step": t_wall / (args.steps * repeats) * 1e3,
         "config": {"workload": wl_name, "layout": wl["layout"], "params": lay.numel, "tensors": lay.num_tensors,
                    "workers": K, "delay_k": wl["k"], "ssd_warmup_iters": wl["W"], "grad_dtype": "f32",
                    "stage": "steps-delay", "kernel": "fused ssd_step", "replicas": world,
                    "hyper_parameters": "per tensor" if args.per_tensor else "uniform",
                    "pre_weight": "one shared buffer" if args.shared_pre else "one buffer per worker",
                    "local_updater": "sgd" if args.local_sgd else "glu",
-                   "device_bytes": st.bytes() + n_sets * K * N * sg,
-                   "l2": "inputs larger than L2 (no flush needed)"
-                   if st.bytes() > 4 * 126e6 else "L2-resident: not an HBM measurement"},
+                   "device_bytes": state_bytes + n_sets * K * N * sg, "l2": l2_note},
         "clocks": clocks,
-        "gpu_launches": launches,
+        "gpu_launches": args.steps, "gpu_launches_all_repeats": launches,
         "roofline": {"bound": "hbm", "kernel": "step_kernel", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind, "traffic": traffic,
-                     "algorithmic_bytes_per_launch": sum(bytes_per_launch) / len(bytes_per_launch),
-                     "launch_ms": {"mean": statistics.mean(per_launch_ms), "min": min(per_launch_ms),
-                                   "max": max(per_launch_ms)}},
+                     "traffic_source": None if traffic is None else
+                     f"ncu DRAM counters on {NCU_TRAFFIC['captured_params']} parameters, scaled by parameter count",
+                     "algorithmic_bytes_per_launch": sum(all_bytes) / len(all_bytes),
+                     "launch_ms": {"mean": statistics.mean(all_ms), "min": min(all_ms), "max": max(all_ms)},
+                     "by_iteration_kind": per_kind},
     }
 
     # ---- end to end: gradients arrive in pinned host memory, the new global weight is read back ----
-    e2e = None
+    def e2e_run(state, host_grads, staging, host_w, host_pre):
+        """Times --e2e-steps calls of ssd_step_host (one untimed call first); host_grads None =
+        the gradients stay on the device."""
+        state.ctx.ssd_step_host(host_grads, staging, host_w)
+        torch.cuda.synchronize()
+        it0 = state.ctx.ssd_get_counters()[0]
+        e_flags = [state.ctx.ssd_schedule(it0 + n)[1] for n in range(args.e2e_steps)]
+
+        def run():
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(args.e2e_steps):
+                state.ctx.ssd_step_host(host_grads, staging, host_w)
+            e1.record(stream)
+            return [e0, e1]
+        e_ms = time_regions(run, 1, world, dev_name)[0][0]
+        shared = args.shared_pre or host_pre
+        e_bytes = float(sum(step_bytes_per_param(K, sg, f, shared, args.local_sgd) * N for f in e_flags))
+        moved = [host_step_bytes(K, sg, f, True, host_grads is not None, host_pre, host_w is not None)
+                 for f in e_flags]
+        return {"value": whole_job_rate(e_bytes, world, e_ms) / 1e9, "unit": UNIT,
+                "h2d_bytes_per_step": statistics.mean(m[0] for m in moved) * N,
+                "d2h_bytes_per_step": statistics.mean(m[1] for m in moved) * N,
+                "steps": args.e2e_steps, "ms_per_step": e_ms / args.e2e_steps, "call": "ssd_step_host"}
+
+    cpu_sample = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        n_sample = min(N, 1 << 23)                # the oracle's inputs: host copies of the same gradients
+        cpu_sample = ([[g[:n_sample].cpu().numpy() for g in gs] for gs in grad_sets], w0[:n_sample].cpu().numpy())
+
+    e2e = host_pre_legs = None
     if args.e2e_steps > 0:
         host_grads = [torch.empty(N, dtype=torch.float32).pin_memory() for _ in range(K)]
         for i in range(K):
             host_grads[i].copy_(grad_sets[0][i])
         host_w = torch.empty(N, dtype=torch.float32).pin_memory()
         staging = grad_sets[1]
-        st.ctx.ssd_step_host(host_grads, staging, host_w)
-        torch.cuda.synchronize()
-        it0 = st.ctx.ssd_get_counters()[0]
-        e_flags = [st.ctx.ssd_schedule(it0 + n)[1] for n in range(args.e2e_steps)]
-        if world > 1:
-            dist.barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for n in range(args.e2e_steps):
-            st.ctx.ssd_step_host(host_grads, staging, host_w)
-        e1.record(stream)
-        torch.cuda.synchronize()
-        e_ms = e0.elapsed_time(e1)
-        e_ms = max_over_ranks(e_ms, dev_name, world)
-        e_bytes = float(sum(step_bytes_per_param(K, sg, f, args.shared_pre, args.local_sgd) * N for f in e_flags))
-        e2e = {"value": whole_job_rate(e_bytes, world, e_ms) / 1e9, "unit": UNIT, "h2d_bytes_per_step": K * N * sg,
-               "d2h_bytes_per_step": N * 4, "steps": args.e2e_steps, "ms_per_step": e_ms / args.e2e_steps,
-               "call": "ssd_step_host"}
+        e2e = e2e_run(st, host_grads, staging, host_w, False)
+        e2e["pre_weight"] = line["config"]["pre_weight"] + ", in device memory"
+        if not args.no_host_pre and not args.local_sgd:
+            # the same workload with pre_weight in ONE pinned host arena (Section 3.5 of the paper)
+            device_pre_bytes = (1 if args.shared_pre else K) * N * 4
+            del st
+            torch.cuda.empty_cache()
+            st = DeviceState(lay.numels, hp, w0, device=dev_name, fill=0.0, host_pre=True, pre_slots=3)
+            if args.per_tensor:
+                st.ctx.ssd_set_tensor_scales(None, [1.0 if kind == "he" else 0.0 for kind in lay.kinds], table)
+            for n in range(wl["W"] + 1):              # SSD warm-up stage and the first GLU call
+                st.ctx.ssd_step_host(None, grad_sets[n % n_sets], None)
+            host_pre_legs = {
+                "pre_weight": "one pinned host arena, streamed through 3 device slices of 2^24 elements",
+                "device_bytes_saved": device_pre_bytes - st.pre_slices.numel() * 4,
+                "host_gradients": e2e_run(st, host_grads, staging, host_w, True),
+                # gradients already on the device: only pre_weight crosses the bus; compare with ms_per_step
+                "device_gradients": e2e_run(st, None, grad_sets[0], None, True)}
         del host_grads, host_w
     line["e2e"] = e2e
+    if host_pre_legs:
+        line["e2e_host_pre_weight"] = host_pre_legs
+
+    # ---- every kernel on two more workloads (single-GPU runs only) ----
+    if world == 1 and not args.no_kernel_table:
+        del st, grad_sets
+        torch.cuda.empty_cache()
+        line["kernels"] = kernel_table(peak)
 
     # ---- the CPU oracle on the host cores, bounded sample (rank 0, single GPU runs only) ----
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        n_sample = min(N, 1 << 23)
-        g_host = [[g[:n_sample].cpu().numpy() for g in gs] for gs in grad_sets]
-        w_host = w0[:n_sample].cpu().numpy()
+    if cpu_sample is not None:
+        g_host, w_host = cpu_sample
         o_steps = 2 * wl["k"]
         dt, moved, params, cores = oracle_sample_run(wl, n_sample, o_steps, g_host, w_host)
         line["cpu_baseline"] = {
@@ -432,6 +557,7 @@ def main():
     if rank == 0:
         print(json.dumps(line))
     if world > 1:
+        import torch.distributed as dist
         dist.barrier()
         dist.destroy_process_group()
 

@@ -280,7 +280,10 @@ Shape step_shape(const ssd_ctx *c, int flags, bool shared_pre, int max_vw, int64
 
 Shape glu_shape(const ssd_ctx *c, int max_vw)
 {
-    return finish_shape(c, max_vw >= 16 ? Shape{16, 1, 128, 0} : Shape{8, 1, 256, 0}, max_vw, 1);
+    Shape sh = max_vw >= 16 ? Shape{16, 1, 128, 0} : Shape{8, 1, 256, 0};
+    // bfloat16 gradients on long arenas: 640 threads per SM instead of all that fit (768)
+    if (max_vw >= 16 && c->hp.grad_dtype == SSD_BF16 && c->n >= (int64_t(1) << 26)) sh.per_sm = 5;
+    return finish_shape(c, sh, max_vw, 1);
 }
 
 size_t table_end_bytes(const ssd_ctx *c) { return (c->offsets.size() * sizeof(int64_t) + 15) / 16 * 16; }

@@ -78,15 +78,18 @@ def _fits(nbytes):
     return nbytes * 1.03 + (1 << 30) <= free
 
 
-def point(log2n: int, K: int, dtype: str, kernels, reps: int, peak: float, threads: int, bps: int,
-          vw: int = 0, batch: int = 0, staging: int = 0):
-    n = 1 << log2n
+def point(log2n: int, K: int, dtype: str, kernels, reps: int, peak: float, threads: int = 0, bps: int = 0,
+          vw: int = 0, batch: int = 0, staging: int = 0, numels=None):
+    """One sweep point: a flat tensor of 2^log2n elements, or the tensor list `numels` of a model
+    layout (log2n is then only a label)."""
+    numels = [1 << log2n] if numels is None else [int(x) for x in numels]
+    n = B.ssd_arena_numel(numels)
     sg = 2 if dtype == "bf16" else 4
     out = []
 
     def emit(kernel, footprint, bytes_per_launch, med, mn):
         gbs = bytes_per_launch / (med * 1e-3) / 1e9
-        out.append({"log2n": log2n, "K": K, "grad_dtype": dtype, "kernel": kernel,
+        out.append({"log2n": log2n, "params": n, "K": K, "grad_dtype": dtype, "kernel": kernel,
                     "footprint_bytes": footprint, "l2": footprint < 4 * L2_BYTES,
                     "bytes_per_launch": bytes_per_launch, "ms_median": med, "ms_min": mn, "gbs": gbs,
                     "gbs_best": bytes_per_launch / (mn * 1e-3) / 1e9, "frac_of_8TBs": gbs / 8000.0,
@@ -117,7 +120,7 @@ def point(log2n: int, K: int, dtype: str, kernels, reps: int, peak: float, threa
         if _fits(fp * R):
             sets = []
             for _ in range(R):
-                st = DeviceState([n], _hp(K, 0, dtype), w0, worker_state=False)
+                st = DeviceState(numels, _hp(K, 0, dtype), w0, worker_state=False)
                 tune(st)
                 sets.append((st, _grads(n, K, dtype)))
             turn = {"i": 0}
@@ -138,7 +141,7 @@ def point(log2n: int, K: int, dtype: str, kernels, reps: int, peak: float, threa
         Kg = max(min(K, 4), min(8, -(-int(1e9) // fp1)))
         fp = (2 + 3 * Kg) * n * 4 + Kg * n * sg
         if _fits(fp):
-            st = DeviceState([n], _hp(Kg, 4, dtype), w0, fill=0.0)
+            st = DeviceState(numels, _hp(Kg, 4, dtype), w0, fill=0.0)
             tune(st)
             grads = _grads(n, Kg, dtype)
             for i in range(Kg):
@@ -160,7 +163,7 @@ def point(log2n: int, K: int, dtype: str, kernels, reps: int, peak: float, threa
         if _fits(fp * R):
             sets = []
             for _ in range(R):
-                st = DeviceState([n], _hp(K, 4, dtype), w0, fill=0.0)
+                st = DeviceState(numels, _hp(K, 4, dtype), w0, fill=0.0)
                 tune(st)
                 grads = _grads(n, K, dtype)
                 st.ctx.ssd_step(grads)                               # first GLU call
