@@ -300,9 +300,9 @@ ssd_status ssd_set_host_chunk(ssd_ctx *ctx, int64_t chunk_elems);
  *                  all K workers, whose pre_weights always hold equal values (see
  *                  "Shared pre_weight" above).  The library reads and writes it;
  *                  its content is part of the state (keep it across a checkpoint).
- *   device_slices  device memory of slots * chunk floats (chunk = the ssd_step_host
- *                  chunk, 2^24 unless changed), 16-byte aligned (32 for the 256-bit
- *                  path), not overlapping any state buffer;
+ *   device_slices  device memory of slots * min(chunk, ssd_arena_numel()) floats
+ *                  (chunk = the ssd_step_host chunk, 2^24 unless changed), 16-byte
+ *                  aligned (32 for the 256-bit path), not overlapping any state buffer;
  *   slots          1..8 slices; 2 or more let the copy of one chunk's slice overlap
  *                  the update of the previous chunk.
  * ssd_step_host then streams pre_weight with the gradients: per chunk, the slice is

@@ -358,6 +358,9 @@ size_t grad_bytes(const ssd_ctx *c) { return static_cast<size_t>(c->n) * (c->hp.
 // stage only through ssd_step_host with a host-resident pre_weight.
 bool lacks_device_pre(const ssd_ctx *c) { return c->hp.local_updater == SSD_LOCAL_GLU && !c->pre_on_device; }
 
+// Elements of one device slice of a host-resident pre_weight: a chunk, or the whole arena if shorter.
+int64_t slice_elems(const ssd_ctx *c) { return c->host_chunk < c->n ? c->host_chunk : c->n; }
+
 ssd_status check_grads(const ssd_ctx *c, const void *const *grads)
 {
     if (!grads) return SSD_ERR_ARG;
@@ -908,7 +911,7 @@ ssd_status ssd_step_host(ssd_ctx *ctx, const void *const *host_grads, void *cons
         const int64_t lo = static_cast<int64_t>(c) * chunk;
         const int64_t count = ctx->n - lo < chunk ? ctx->n - lo : chunk;
         const int slot = host_pre ? c % slots : 0;
-        float *slice = host_pre ? ctx->pre_slices + static_cast<int64_t>(slot) * chunk : nullptr;
+        float *slice = host_pre ? ctx->pre_slices + static_cast<int64_t>(slot) * slice_elems(ctx) : nullptr;
         cudaEvent_t ev_slot = ctx->events[ev_slot_at + slot];
         // the slice is free once the chunk that used it last (c - slots) is done with it
         if (host_pre && c >= slots) e = cudaStreamWaitEvent(ctx->in_stream, ev_slot, 0);
@@ -970,7 +973,7 @@ ssd_status ssd_set_host_pre_weight(ssd_ctx *ctx, float *host_pre, float *device_
     if (!host_pre || !device_slices || slots < 1 || slots > kMaxPreSlots) return SSD_ERR_ARG;
     if (!ctx->has_workers || ctx->hp.delay_k == 0 || ctx->pre_on_device) return SSD_ERR_STATE;
     if (!aligned16(host_pre) || !aligned16(device_slices)) return SSD_ERR_ALIGN;
-    const size_t bytes = static_cast<size_t>(slots) * static_cast<size_t>(ctx->host_chunk) * sizeof(float);
+    const size_t bytes = static_cast<size_t>(slots) * static_cast<size_t>(slice_elems(ctx)) * sizeof(float);
     if (touches_state(ctx, device_slices, bytes)) return SSD_ERR_ARG;
     ctx->host_pre = host_pre;
     ctx->pre_slices = device_slices;

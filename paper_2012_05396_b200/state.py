@@ -109,7 +109,7 @@ class DeviceState:
             self.ctx = B.Context(self.numels, hp, self.w, self.mom, self.w_loc, None, self.w_dev)
             if host_chunk:
                 self.ctx.ssd_set_host_chunk(host_chunk)
-            chunk = host_chunk or (1 << 24)
+            chunk = min(host_chunk or (1 << 24), self.n)
             slices = ArenaSlab(1, pre_slots * chunk, torch.float32, self.device)
             self.slabs.append(slices)
             self.pre_slices = slices.arenas[0]
