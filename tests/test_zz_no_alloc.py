@@ -91,12 +91,13 @@ def test_static_table_update_against_the_cpu_oracle(bf16):
         if call < 2:
             dev.ctx.ssd_server_sync_update_static(grads, lr_mult, wd_mult)
             ohp.set_tensor_scales(ends, lr_mult, wd_mult)
+            if call == 1:                                    # (the first call did the one-time address look-up)
+                torch.cuda.synchronize()
+                assert torch.cuda.mem_get_info()[0] >= free_before, "the warm call took device memory"
         else:                                                # the ordinary call still uses the context's own table
             dev.ctx.ssd_server_sync_update(grads)
             ohp.set_tensor_scales(ends, own_lr, own_wd)
         torch.cuda.synchronize()
-        if call == 1:                                        # (the first call did the one-time address look-up)
-            assert torch.cuda.mem_get_info()[0] == free_before, "the warm call changed the free device memory"
         oracle.server_update(ohp, [oracle_grad(g, bf16) for g in grads], ref_w, ref_mom)
         assert_same(dev.w, ref_w, f"w after call {call}")
         assert_same(dev.mom, ref_mom, f"mom after call {call}")
