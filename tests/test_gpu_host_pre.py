@@ -148,3 +148,36 @@ def test_host_pre_weight_survives_a_checkpoint():
     for n in range(6, 13):
         ref.step([h.numpy() for h in step(b, n)])
     compare_states(b, ref, "resumed")
+
+
+def test_plain_sgd_updater_needs_no_pre_weight_at_all():
+    # Eq. 5 as local updater never touches pre_weight: a context created without pre_weight buffers (and
+    # without a host arena) runs every delay-stage call, fused, split and through the host pipeline
+    lay = synth.get_layout("resnet20")
+    K, W, k = 3, 1, 2
+    ohp, chp = make_hp(K, 0.1, 0.9, W, k, wd=1e-3, lr_loc=0.25, local_sgd=True)
+    w0 = synth.init_weights(lay)
+    full = DeviceState(lay.numels, chp, w0)                    # only for its arenas
+    ctx = B.Context(lay.numels, chp, full.w, full.mom, full.w_loc, None, full.w_dev)
+    ref = oracle.State(ohp, w0.numpy())
+    staging = [torch.empty(full.n, dtype=torch.float32, device="cuda") for _ in range(K)]
+    for n in range(9):
+        grads = [synth.gradient(lay, n, i, 1e-2, device="cuda") for i in range(K)]
+        if n % 3 == 0:
+            ctx.ssd_step(grads)
+        elif n % 3 == 1:
+            ctx.ssd_server_sync_update(grads)
+            for i in range(K):
+                ctx.ssd_worker_local_step(i, grads[i])
+            ctx.ssd_advance()
+        else:
+            host = [pinned(g) for g in grads]
+            ctx.ssd_step_host(host, staging, None)
+        torch.cuda.synchronize()
+        ref.step([g.cpu().numpy() for g in grads])
+    assert_same(full.w, ref.w, "w")
+    assert_same(full.mom, ref.mom, "mom")
+    for i in range(K):
+        assert_same(full.w_loc[i], ref.w_loc[i], f"w_loc[{i}]")
+        assert_same(full.w_dev[i], ref.w_dev[i], f"w_dev[{i}]")
+    assert full.guards_intact()

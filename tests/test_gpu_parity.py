@@ -256,6 +256,14 @@ def test_every_kernel_shape_and_alignment_gives_the_same_bits(bf16):
                 gpu_iteration(dev, gs, mode)
             torch.cuda.synchronize()
             compare_states(dev, ref, f"shape vw={vw} batch={batch} {mode}")
+    # a thread count above what the 16-element kernels are compiled for is brought down, not refused
+    dev = DeviceState(lay.numels, chp, w0)
+    dev.ctx.ssd_set_kernel_shape(16, 2)
+    dev.ctx.ssd_set_launch(512, 1)
+    for gs in grads:
+        gpu_iteration(dev, gs, "fused")
+    torch.cuda.synchronize()
+    compare_states(dev, ref, "vw=16 with 512 threads asked")
     # misaligned gradient buffers (float32 only matters) and misaligned state
     shift = 8 if bf16 else 4
     dev = DeviceState(lay.numels, chp, w0)
@@ -562,6 +570,50 @@ def test_random_combinations_of_every_option():
             ref.step([oracle_grad(g, bf16) for g in grads])
         torch.cuda.synchronize()
         compare_states(dev, ref, tag)
+
+
+def test_fused_steps_replayed_from_a_cuda_graph():
+    # one period of k delay-stage iterations captured into a CUDA graph and replayed for later periods,
+    # the gradients written into the same buffers before each replay; the counters are set by hand
+    K, W, k, periods = 4, 2, 4, 3
+    lay = synth.get_layout("resnet20")
+    ohp, chp = make_hp(K, 0.1, 0.9, W, k, wd=1e-3)
+    w0 = synth.init_weights(lay)
+    dev = DeviceState(lay.numels, chp, w0)
+    ref = oracle.State(ohp, w0.numpy())
+    slots = [[torch.empty(dev.n, dtype=torch.float32, device="cuda") for _ in range(K)] for _ in range(k)]
+
+    def fill(n, j):
+        grads = [synth.gradient(lay, n, i, 1e-2, device="cuda") for i in range(K)]
+        for s, g in zip(slots[j], grads):
+            s.copy_(g)
+        ref.step([g.cpu().numpy() for g in grads])
+
+    n = 0
+    for _ in range(W + 1 + k):                     # warm-up, first GLU call, one whole period outside capture
+        fill(n, n % k)
+        dev.ctx.ssd_step(slots[n % k])
+        n += 1
+    torch.cuda.synchronize()
+    compare_states(dev, ref, "before capture")
+    base = n
+    # capture the next period (its launches do not run now: the state is untouched, the counters move)
+    graph, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+    it0, lu0, _, _ = dev.ctx.ssd_get_counters()
+    with torch.cuda.graph(graph, stream=side):
+        for j in range(k):
+            dev.ctx.ssd_step(slots[(base + j) % k])
+    assert dev.ctx.ssd_get_counters()[:2] == (it0 + k, lu0 + k)
+    dev.ctx.ssd_set_counters(it0, lu0)
+    for p in range(periods):
+        for j in range(k):
+            fill(n, n % k)
+            n += 1
+        graph.replay()
+        it, lu, _, _ = dev.ctx.ssd_get_counters()
+        dev.ctx.ssd_set_counters(it + k, lu + k)
+        torch.cuda.synchronize()
+        compare_states(dev, ref, f"after replay {p}")
 
 
 @pytest.mark.parametrize("bf16", [False, True])
