@@ -181,3 +181,83 @@ def test_plain_sgd_updater_needs_no_pre_weight_at_all():
         assert_same(full.w_loc[i], ref.w_loc[i], f"w_loc[{i}]")
         assert_same(full.w_dev[i], ref.w_dev[i], f"w_dev[{i}]")
     assert full.guards_intact()
+
+
+def test_random_host_pipelines():
+    # seeded draw over arena sizes, chunk sizes, slice counts, schedules, gradient types and where the
+    # gradients and pre_weight live; every iteration compared with the oracle
+    rng = np.random.default_rng(35)
+    for case in range(16):
+        T = int(rng.integers(1, 6))
+        numels = [int(rng.choice([3, 100, 1000, 4099, 30000, 70001])) for _ in range(T)]
+        K = int(rng.choice([1, 2, 3, 5, 8]))
+        W, k = int(rng.integers(0, 3)), int(rng.integers(1, 5))
+        bf16, host_pre, host_grads = bool(rng.integers(2)), bool(rng.integers(3) > 0), bool(rng.integers(2))
+        chunk = int(rng.choice([1024, 4096, 1 << 15, 1 << 17]))
+        slots = int(rng.integers(1, 5))
+        lay = synth.Layout("t")
+        for i, cnt in enumerate(numels):
+            lay.add(f"x{i}", cnt, "he", 8)
+        tag = f"case {case}: numels={numels} K={K} W={W} k={k} bf16={bf16} host_pre={host_pre} " \
+              f"host_grads={host_grads} chunk={chunk} slots={slots}"
+        ohp, chp = make_hp(K, 0.1, 0.9, W, k, wd=0.01, bf16=bf16)
+        w0 = synth.init_weights(lay, seed=case)
+        dev = DeviceState(lay.numels, chp, w0, host_pre=host_pre, pre_slots=slots, host_chunk=chunk)
+        if not host_pre:
+            dev.ctx.ssd_set_host_chunk(chunk)
+        ref = oracle.State(ohp, w0.numpy())
+        gdtype = torch.bfloat16 if bf16 else torch.float32
+        staging = [torch.empty(dev.n, dtype=gdtype, device="cuda") for _ in range(K)]
+        w_out = torch.empty(dev.n, dtype=torch.float32).pin_memory()
+        for n in range(W + 2 * k + 2):
+            grads = [synth.gradient(lay, n, i, 0.05, seed=case, device="cuda") for i in range(K)]
+            if bf16:
+                grads = [synth.to_bf16(g) for g in grads]
+            if host_grads:
+                host = [pinned(g) for g in grads]
+                dev.ctx.ssd_step_host(host, staging, w_out)
+            else:
+                for s, g in zip(staging, grads):
+                    s.copy_(g)
+                dev.ctx.ssd_step_host(None, staging, w_out)
+            ref.step([oracle_grad(g, bf16) for g in grads])
+            torch.cuda.synchronize()
+            assert_same(w_out, ref.w, f"{tag} iter {n} w read back")
+            compare_states(dev, ref, f"{tag} iter {n}")
+
+
+def test_two_contexts_on_two_host_threads_and_streams():
+    # a context is used by one host thread at a time; two threads with a context and a stream each run
+    # their schedules concurrently and neither disturbs the other
+    import threading
+    lay = synth.get_layout("resnet56")
+    K, W, k, iters = 3, 1, 2, 12
+    results, errors = {}, []
+
+    def work(tid):
+        try:
+            torch.cuda.set_device(0)
+            ohp, chp = make_hp(K, 0.1, 0.9, W, k, wd=1e-3 * (tid + 1))
+            w0 = synth.init_weights(lay, seed=100 + tid)
+            stream = torch.cuda.Stream()
+            with torch.cuda.stream(stream):
+                dev = DeviceState(lay.numels, chp, w0)
+                ref = oracle.State(ohp, w0.numpy())
+                for n in range(iters):
+                    grads = [synth.gradient(lay, n, i, 1e-2, seed=100 + tid, device="cuda") for i in range(K)]
+                    dev.ctx.ssd_step(grads, stream=stream)
+                    ref.step([g.cpu().numpy() for g in grads])
+                stream.synchronize()
+            results[tid] = (dev, ref)
+        except Exception as exc:                      # surfaced in the main thread below
+            errors.append(exc)
+
+    threads = [threading.Thread(target=work, args=(t,)) for t in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    torch.cuda.synchronize()
+    for tid, (dev, ref) in results.items():
+        compare_states(dev, ref, f"thread {tid}")
