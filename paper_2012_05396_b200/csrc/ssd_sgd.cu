@@ -383,15 +383,15 @@ int even_batch(int K, int batch)
 template <int GT, int VW, bool PT>
 ssd_status launch_sync_b(ssd_ctx *c, SyncParams &p, const Shape &sh, cudaStream_t stream)
 {
-    const int compiled = sh.batch >= 8 ? ((VW == 16 && GT == kF32) ? 4 : 8) : sh.batch >= 4 ? 4 : sh.batch >= 2 ? 2 : 1;
-    p.per_batch = even_batch(p.K, compiled);
-    switch (sh.batch) {
+    // eight float32 vectors of 16 in flight would spill: four is the most there
+    constexpr int kMost = (VW == 16 && GT == kF32) ? 4 : 8;
+    const int batch = sh.batch < kMost ? sh.batch : kMost;
+    p.per_batch = even_batch(p.K, batch);
+    switch (batch) {
     case 1: return launch(c, sync_kernel<GT, VW, 1, PT>, p, p.n, sh, stream);
     case 2: return launch(c, sync_kernel<GT, VW, 2, PT>, p, p.n, sh, stream);
     case 4: return launch(c, sync_kernel<GT, VW, 4, PT>, p, p.n, sh, stream);
-    default:
-        // eight float32 vectors of 16 in flight would spill: four is the most there
-        return launch(c, sync_kernel<GT, VW, (VW == 16 && GT == kF32) ? 4 : 8, PT>, p, p.n, sh, stream);
+    default: return launch(c, sync_kernel<GT, VW, kMost, PT>, p, p.n, sh, stream);
     }
 }
 
@@ -412,8 +412,9 @@ const void *grad_at(const ssd_ctx *c, const void *g, int64_t lo)
     return static_cast<const unsigned char *>(g) + lo * (c->hp.grad_dtype == SSD_BF16 ? 2 : 4);
 }
 
-// The launch functions take an element range [lo, lo + count) of the arena (lo a multiple of 8,
-// which keeps every alignment property of the buffers); count < 0 means the whole arena.
+// The launch functions take an element range [lo, lo + count) of the arena (lo a multiple of 4, as
+// tensor offsets are; max_vector narrows the accesses where lo shifts a buffer's alignment);
+// count < 0 means the whole arena.
 ssd_status launch_sync(ssd_ctx *c, const void *const *grads, int flags, cudaStream_t stream,
                        int64_t lo = 0, int64_t count = -1)
 {
@@ -468,12 +469,15 @@ ssd_status launch_glu(ssd_ctx *c, int worker, const void *grad, int flags, cudaS
 template <int GT, int VW, bool PT>
 ssd_status launch_step_b(ssd_ctx *c, StepParams &p, const Shape &sh, cudaStream_t stream)
 {
-    p.per_batch = even_batch(p.K, sh.batch == 1 ? 1 : (sh.batch == 2 || VW >= 8) ? 2 : 4);
-    // step_shape keeps the batch at 2 or below for vectors of 8 and more (4 would spill)
-    if (sh.batch == 1) return launch(c, step_kernel<GT, VW, 1, PT>, p, p.n, sh, stream);
-    if constexpr (VW == 4)
-        if (sh.batch > 2) return launch(c, step_kernel<GT, 4, 4, PT>, p, p.n, sh, stream);
-    return launch(c, step_kernel<GT, VW, 2, PT>, p, p.n, sh, stream);
+    // step_shape keeps the batch at 2 or below for vectors of 8 and 16 (4 would spill)
+    constexpr int kMost = VW == 4 ? 4 : 2;
+    const int batch = sh.batch < kMost ? sh.batch : kMost;
+    p.per_batch = even_batch(p.K, batch);
+    switch (batch) {
+    case 1: return launch(c, step_kernel<GT, VW, 1, PT>, p, p.n, sh, stream);
+    case 2: return launch(c, step_kernel<GT, VW, 2, PT>, p, p.n, sh, stream);
+    default: return launch(c, step_kernel<GT, VW, kMost, PT>, p, p.n, sh, stream);
+    }
 }
 
 template <bool PT>
