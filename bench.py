@@ -62,14 +62,20 @@ def kernel_digest() -> str:
     return h.hexdigest()[:16]
 
 
-def step_bytes_per_param(K: int, sg: int, flags: int, shared_pre: bool = False, local_sgd: bool = False) -> int:
+def step_bytes_per_param(K: int, sg: int, flags: int, shared_pre: bool = False, local_sgd: bool = False,
+                         merged_dev: bool = False) -> int:
     """Algorithmic bytes one fused delay-stage step moves per parameter: K gradients, K local
     weights read and written, K pre_weights read, w and mom read and written; a refresh adds K
     pre_weight stores, a pull adds K device-weight stores (and trades nothing else).  With one
-    shared pre_weight buffer it is read once and refreshed once instead of K times."""
+    shared pre_weight buffer it is read once and refreshed once instead of K times.  Without
+    separate device weights (merged_dev) a pull iteration is the server update plus K stores of the
+    new global weight (plus, where it also writes pre_weight, the old local weights going there)."""
+    pre_copies = 1 if shared_pre else K
+    if merged_dev and flags & 4:
+        writes_pre = bool(flags & 3) and not local_sgd
+        return K * sg + 16 + 4 * K + (8 * pre_copies if writes_pre else 0)
     if local_sgd:       # plain-SGD local updater: no pre_weight traffic at all
         return K * (sg + 8) + 16 + (4 * K if flags & 4 else 0)
-    pre_copies = 1 if shared_pre else K
     b = K * (sg + 8) + 4 * pre_copies + 16
     if flags & 2:       # refresh
         b += 4 * pre_copies
@@ -289,7 +295,7 @@ def kernel_table(peak: float):
     cases = [("resnet50_K8_f32", synth.get_layout("resnet50").numels, 25, 8, "f32"),
              ("flat2p26_K16_bf16", None, 26, 16, "bf16")]
     for name, numels, log2n, K, dtype in cases:
-        for rec in sweep.point(log2n, K, dtype, ["sync", "glu", "step"], 20, peak, numels=numels):
+        for rec in sweep.point(log2n, K, dtype, ["sync", "glu", "step", "step_merged"], 20, peak, numels=numels):
             if "gbs" not in rec:
                 rows.append({"workload": name, "kernel": rec["kernel"], "skipped": rec.get("skipped")})
                 continue
@@ -319,6 +325,8 @@ def main():
                     help="per-tensor hyper-parameters: weight decay 5e-4 on conv/FC weights only")
     ap.add_argument("--shared-pre", action="store_true",
                     help="one pre_weight buffer shared by all workers (fewer algorithmic bytes, counted as such)")
+    ap.add_argument("--merged-dev", action="store_true",
+                    help="no separate device weights (w_dev[i] is w_loc[i]): pull iterations skip the local update")
     ap.add_argument("--local-sgd", action="store_true",
                     help="workers update with plain SGD (Eq. 5) instead of GLU (fewer algorithmic bytes, counted as such)")
     ap.add_argument("--threads", type=int, default=0, help="threads per block (0 = library default)")
@@ -362,7 +370,8 @@ def main():
                         lr_local=nan, alpha=nan, beta=nan, rescale=nan, grad_dtype=B.SSD_F32,
                         local_updater=B.SSD_LOCAL_SGD if args.local_sgd else B.SSD_LOCAL_GLU)
     w0 = synth.init_weights(lay, device=dev_name)
-    st = DeviceState(lay.numels, hp, w0, device=dev_name, fill=0.0, shared_pre=args.shared_pre)
+    st = DeviceState(lay.numels, hp, w0, device=dev_name, fill=0.0, shared_pre=args.shared_pre,
+                     merged_dev=args.merged_dev)
     if args.per_tensor:
         table = torch.empty(st.ctx.ssd_tensor_table_bytes(), dtype=torch.uint8, device=dev_name)
         st.ctx.ssd_set_tensor_scales(None, [1.0 if kind == "he" else 0.0 for kind in lay.kinds], table)
@@ -417,7 +426,7 @@ def main():
     launches = st.ctx.ssd_kernel_launches() - launches0
 
     def region_bytes(flags):
-        return [step_bytes_per_param(K, sg, f, args.shared_pre, args.local_sgd) * N for f in flags]
+        return [step_bytes_per_param(K, sg, f, args.shared_pre, args.local_sgd, args.merged_dev) * N for f in flags]
 
     rates = [whole_job_rate(float(sum(region_bytes(f))), world, ms) / 1e9
              for f, (ms, _) in zip(flags_per_region, regions)]
@@ -436,11 +445,12 @@ def main():
             by_flags.setdefault(fl & 6, []).append(ms)
     names = {0: "plain", 2: "refresh", 4: "pull", 6: "refresh+pull"}
     per_kind = {names[fl]: {"launches": len(ms), "ms_median": statistics.median(ms),
-                            "gbs": step_bytes_per_param(K, sg, fl, args.shared_pre, args.local_sgd) * N
+                            "gbs": step_bytes_per_param(K, sg, fl, args.shared_pre, args.local_sgd, args.merged_dev) * N
                             / (statistics.median(ms) * 1e-3) / 1e9}
                 for fl, ms in sorted(by_flags.items())}
     traffic = None
-    plain_config = not (args.shared_pre or args.local_sgd or args.per_tensor or args.threads or args.blocks_per_sm)
+    plain_config = not (args.shared_pre or args.local_sgd or args.per_tensor or args.threads or args.blocks_per_sm
+                        or args.merged_dev)
     if NCU_TRAFFIC["digest"] == kernel_digest() and NCU_TRAFFIC["K"] == K and plain_config:
         per = NCU_TRAFFIC["bytes_per_param"]
         kinds = [f & 6 for fl in flags_per_region for f in fl]
@@ -462,10 +472,13 @@ def main():
                    "hyper_parameters": "per tensor" if args.per_tensor else "uniform",
                    "pre_weight": "one shared buffer" if args.shared_pre else "one buffer per worker",
                    "local_updater": "sgd" if args.local_sgd else "glu",
+                   "device_weights": "the local weights (no separate buffers)" if args.merged_dev
+                   else "one buffer per worker",
                    "device_bytes": state_bytes + n_sets * K * N * sg, "l2": l2_note},
         "clocks": clocks,
         "gpu_launches": args.steps, "gpu_launches_all_repeats": launches,
-        "roofline": {"bound": "hbm", "kernel": "step_kernel", "achieved": achieved, "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": "step_kernel (pull iterations: sync_kernel)" if args.merged_dev
+                     else "step_kernel", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind, "traffic": traffic,
                      "traffic_source": None if traffic is None else
                      f"ncu DRAM counters on {NCU_TRAFFIC['captured_params']} parameters, scaled by parameter count",

@@ -137,7 +137,19 @@ typedef struct {
  * once per element instead of K times and writes it once (K-1 arenas less memory,
  * 4(K-1) bytes per parameter less traffic); results are unchanged.  The per-worker
  * calls (ssd_worker_glu_update, ssd_worker_local_step in the delay stage) would
- * overwrite it between workers and return SSD_ERR_STATE for such a context. */
+ * overwrite it between workers and return SSD_ERR_STATE for such a context.
+ * Merged device weights: w_dev[i] == w_loc[i] for every worker (all of them or none:
+ * SSD_ERR_ARG otherwise) declares that the caller keeps no separate device weights.
+ * Algorithm 1 hands the local update's result to the devices on a pull iteration and
+ * then overwrites the local weight with the pulled global weight; with one buffer for
+ * both, that result is overwritten before anyone could read it, so on pull iterations
+ * the local update is skipped altogether: w_loc[i] = w (after pre_weight = old
+ * w_loc[i], where the iteration writes pre_weight), and the next gradient is computed
+ * on the pulled weight.  w, mom, w_loc and pre_weight are, bit for bit, what the
+ * separate-buffer form gives, on every iteration; only the device-weight output of
+ * pull iterations is not produced.  K arenas less memory; a fused pull iteration
+ * moves K*(sg+4)+16 bytes per parameter instead of K*(sg+16)+16 (sg = bytes per
+ * gradient element). */
 typedef struct {
     float *w;                     /* global weight w_t (server)                 */
     float *mom;                   /* server momentum mom_t                      */
@@ -344,7 +356,8 @@ ssd_status ssd_broadcast_weights(ssd_ctx *ctx, void *cuda_stream);
 
 /* Where worker `worker` finds the weights for its next forward/backward pass
  * after the iterations done so far: the global w in the warm-up stage, w_loc_i
- * after a GLU step without pull, w_dev_i after a pull iteration.  `view`
+ * after a GLU step without pull, w_dev_i after a pull iteration (w_loc_i, which
+ * then holds the pulled weight, for a context with merged device weights).  `view`
  * receives the SSD_VIEW_* code; either output may be NULL. */
 ssd_status ssd_worker_weights(const ssd_ctx *ctx, int32_t worker, const float **weights,
                               int32_t *view);

@@ -28,7 +28,11 @@ namespace ssd {
 constexpr int kMaxWorkers = 32;
 constexpr int kMaxThreads = 512;   // upper bound of threads per block for every kernel here
 
-enum : int { kFirst = 1, kRefresh = 2, kPull = 4, kCopy = 8, kLocalSgd = 16 };   // kLocalSgd: internal
+// kLocalSgd, kMergedDev: internal.  kMergedDev: the workers' device weights are the same buffers as
+// their local weights, so on a pull iteration the local update's result has nowhere to go (the
+// pulled global weight overwrites it at once) and is neither computed nor stored; such iterations
+// run the *_merged_pull kernels instead of glu_kernel / step_kernel.
+enum : int { kFirst = 1, kRefresh = 2, kPull = 4, kCopy = 8, kLocalSgd = 16, kMergedDev = 32 };
 enum : int { kF32 = 0, kBF16 = 1 };
 
 struct Scalars {
@@ -354,6 +358,55 @@ __device__ __forceinline__ void glu_at(const GluParams &p, int64_t e)
     }
 }
 
+// One worker's pull when its device weights are its local weights (kMergedDev): pre_weight takes
+// the old local weight where the iteration writes pre_weight, the local weight takes the global one.
+template <int VW> __device__ __forceinline__ void glu_merged_pull_at(const GluParams &p, int64_t e)
+{
+    const bool writes_pre = (p.flags & (kFirst | kRefresh)) && !(p.flags & kLocalSgd);
+    Vec<VW> wg = ld_f32<VW>(p.w, e);
+    if (writes_pre) st_f32<VW>(p.pre, e, ld_f32<VW>(p.w_loc, e));
+    st_f32<VW>(p.w_loc, e, wg);
+}
+
+// Pull iteration of a context whose device weights are its local weights (kMergedDev): the
+// server update, pre_weight = old local weight where the iteration writes pre_weight (only with
+// k = 1 does a pull coincide with that), then every local weight takes the new global weight.
+// The local update itself is skipped: its result would be overwritten before anyone could read it.
+template <int GT, int VW, int B, bool PT>
+__device__ __forceinline__ void step_merged_pull_at(const StepParams &p, int64_t e)
+{
+    const bool sgd = p.flags & kLocalSgd;
+    const bool writes_pre = (p.flags & (kFirst | kRefresh)) && !sgd;
+    Vec<VW> w = ld_f32<VW>(p.w, e);
+    Vec<VW> mom = ld_f32<VW>(p.mom, e);
+    Vec<VW> sum;
+    const int per = p.per_batch;
+    for (int i0 = 0; i0 < p.K; i0 += per) {
+        Grad<GT, VW> g[B];
+#pragma unroll
+        for (int b = 0; b < B; ++b)
+            if (b < per && i0 + b < p.K) g[b] = ld_grad<GT, VW>(p.g[i0 + b], e);
+#pragma unroll
+        for (int b = 0; b < B; ++b) {
+            if (b < per && i0 + b < p.K) {
+#pragma unroll
+                for (int l = 0; l < VW; ++l)
+                    sum.v[l] = (i0 + b == 0) ? g[b].get(l) : __fadd_rn(sum.v[l], g[b].get(l));
+            }
+        }
+    }
+    const GroupScalars<PT, VW> sc(p.s, p.tt, e);
+#pragma unroll
+    for (int l = 0; l < VW; ++l) server_elem(sum.v[l], w.v[l], mom.v[l], sc.at(l));
+    if (writes_pre) {
+        const int copies = p.shared_pre ? 1 : p.K;
+        for (int i = 0; i < copies; ++i) st_f32<VW>(p.pre[i], e, ld_f32<VW>(p.w_loc[i], e));
+    }
+    st_f32<VW>(p.mom, e, mom);
+    st_f32<VW>(p.w, e, w);
+    for (int i = 0; i < p.K; ++i) st_f32<VW>(p.w_loc[i], e, w);
+}
+
 template <int GT, int VW, int B, bool PT>
 __device__ __forceinline__ void step_at(const StepParams &p, int64_t e)
 {
@@ -446,6 +499,20 @@ template <int GT, int VW, int B, bool PT>
 __global__ void __launch_bounds__(threads_bound(VW)) step_kernel(const __grid_constant__ StepParams p)
 {
     SSD_SWEEP(p.n, VW, (step_at<GT, VW, B, PT>(p, e)), (step_at<GT, 4, B, PT>(p, e)));
+}
+
+// The two pull forms of a context with merged device weights, as kernels of their own so that the
+// kernels above keep their register budgets.
+template <int GT, int VW, int B, bool PT>
+__global__ void __launch_bounds__(threads_bound(VW)) step_merged_pull_kernel(const __grid_constant__ StepParams p)
+{
+    SSD_SWEEP(p.n, VW, (step_merged_pull_at<GT, VW, B, PT>(p, e)), (step_merged_pull_at<GT, 4, B, PT>(p, e)));
+}
+
+template <int VW>
+__global__ void __launch_bounds__(threads_bound(VW)) glu_merged_pull_kernel(const __grid_constant__ GluParams p)
+{
+    SSD_SWEEP(p.n, VW, (glu_merged_pull_at<VW>(p, e)), (glu_merged_pull_at<4>(p, e)));
 }
 
 template <int VW> __device__ __forceinline__ void copy_at(const CopyParams &p, int64_t e)

@@ -47,6 +47,7 @@ struct ssd_ctx {
     bool has_workers = true;          // false: delay_k == 0 and no worker tables were given
     bool shared_pre = false;          // all K pre_weight pointers are the same buffer
     bool pre_on_device = true;        // false: created without pre_weight buffers (see ssd_set_host_pre_weight)
+    bool merged_dev = false;          // w_dev[i] == w_loc[i] for every worker: no separate device weights
     // pre_weight kept in host memory: one pinned host arena, streamed through `pre_slots` device
     // slices of `host_chunk` elements by ssd_step_host
     float *host_pre = nullptr, *pre_slices = nullptr;
@@ -224,10 +225,18 @@ Shape finish_shape(const ssd_ctx *c, Shape sh, int max_vw, int max_batch)
 // reads and writes: too few bytes in flight cannot cover the DRAM latency, too many lower
 // the DRAM efficiency again, sooner so when a large share of the traffic is writes.  The
 // values below are the measured optima on B200 (arenas of 25M..138M elements).
-Shape sync_shape(const ssd_ctx *c, int max_vw)
+Shape sync_shape(const ssd_ctx *c, int max_vw, int flags = 0)
 {
     const int K = c->hp.K;
     Shape sh;
+    if (flags & kCopy) {
+        // K + 2 stores per element behind the K + 2 loads (the hand-over iteration of the warm-up
+        // stage, and every pull of a context with merged device weights): 44 % of the traffic is
+        // writes, and 384 threads per SM is the optimum whatever K (6.5-6.65 TB/s float32,
+        // 6.25-6.5 bfloat16, against 5.9-6.1 with the shapes below)
+        const bool wide = c->hp.grad_dtype == SSD_BF16 && max_vw >= 16;
+        return finish_shape(c, wide ? Shape{16, 2, 128, 3} : Shape{8, 4, 128, 3}, max_vw, 8);
+    }
     // (the batch is an upper bound: the K workers go in ceil(K / batch) batches of equal size)
     if (c->hp.grad_dtype == SSD_BF16) {
         // bfloat16 gradients: vectors of 16 fetch them with 256-bit loads like the float32 state
@@ -432,7 +441,7 @@ ssd_status launch_sync(ssd_ctx *c, const void *const *grads, int flags, cudaStre
     const bool state32 = (flags & kCopy) ? c->state32 : (aligned32(c->w) && aligned32(c->mom));
     p.tt = table_of(c);
     p.tt.base = lo;
-    const Shape sh = sync_shape(c, max_vector(c, state32, grads, c->hp.K, lo));
+    const Shape sh = sync_shape(c, max_vector(c, state32, grads, c->hp.K, lo), flags);
     return p.tt.T ? launch_sync_t<true>(c, p, sh, stream) : launch_sync_t<false>(c, p, sh, stream);
 }
 
@@ -462,6 +471,13 @@ ssd_status launch_glu(ssd_ctx *c, int worker, const void *grad, int flags, cudaS
     p.flags = flags | (c->hp.local_updater == SSD_LOCAL_SGD ? kLocalSgd : 0);
     p.s = c->s;
     p.tt = table_of(c);
+    if (c->merged_dev && (flags & kPull)) {
+        // no separate device weights: the pull is all that is left of this worker's iteration
+        p.flags |= kMergedDev;
+        const Shape sh = finish_shape(c, Shape{8, 1, 256, 0}, c->state32 ? 8 : 4, 1);
+        if (sh.vw == 8) return launch(c, glu_merged_pull_kernel<8>, p, p.n, sh, stream);
+        return launch(c, glu_merged_pull_kernel<4>, p, p.n, sh, stream);
+    }
     const Shape sh = glu_shape(c, max_vector(c, c->state32, &grad, 1, 0));
     return p.tt.T ? launch_glu_t<true>(c, p, sh, stream) : launch_glu_t<false>(c, p, sh, stream);
 }
@@ -489,6 +505,33 @@ ssd_status launch_step_t(ssd_ctx *c, StepParams &p, const Shape &sh, cudaStream_
     if (sh.vw == 8)
         return bf16 ? launch_step_b<kBF16, 8, PT>(c, p, sh, stream) : launch_step_b<kF32, 8, PT>(c, p, sh, stream);
     return bf16 ? launch_step_b<kBF16, 4, PT>(c, p, sh, stream) : launch_step_b<kF32, 4, PT>(c, p, sh, stream);
+}
+
+// Pull iteration that also writes pre_weight (k = 1) of a context with merged device weights; the
+// loads are the server kernel's, so it takes the server kernel's shape and batches.
+template <int GT, int VW, bool PT>
+ssd_status launch_merged_pull_b(ssd_ctx *c, StepParams &p, const Shape &sh, cudaStream_t stream)
+{
+    constexpr int kMost = (VW == 16 && GT == kF32) ? 4 : 8;
+    const int batch = sh.batch < kMost ? sh.batch : kMost;
+    p.per_batch = even_batch(p.K, batch);
+    switch (batch) {
+    case 1: return launch(c, step_merged_pull_kernel<GT, VW, 1, PT>, p, p.n, sh, stream);
+    case 2: return launch(c, step_merged_pull_kernel<GT, VW, 2, PT>, p, p.n, sh, stream);
+    case 4: return launch(c, step_merged_pull_kernel<GT, VW, 4, PT>, p, p.n, sh, stream);
+    default: return launch(c, step_merged_pull_kernel<GT, VW, kMost, PT>, p, p.n, sh, stream);
+    }
+}
+
+template <bool PT>
+ssd_status launch_merged_pull_t(ssd_ctx *c, StepParams &p, const Shape &sh, cudaStream_t stream)
+{
+    const bool bf16 = c->hp.grad_dtype == SSD_BF16;
+    if (sh.vw == 16)
+        return bf16 ? launch_merged_pull_b<kBF16, 16, PT>(c, p, sh, stream) : launch_merged_pull_b<kF32, 16, PT>(c, p, sh, stream);
+    if (sh.vw == 8)
+        return bf16 ? launch_merged_pull_b<kBF16, 8, PT>(c, p, sh, stream) : launch_merged_pull_b<kF32, 8, PT>(c, p, sh, stream);
+    return bf16 ? launch_merged_pull_b<kBF16, 4, PT>(c, p, sh, stream) : launch_merged_pull_b<kF32, 4, PT>(c, p, sh, stream);
 }
 
 // The shared-memory ring covers the common case; the rest stays on the register path.  Its bulk
@@ -535,6 +578,11 @@ ssd_status launch_step_ring(ssd_ctx *c, const StepParams &p, cudaStream_t stream
 ssd_status launch_step(ssd_ctx *c, const void *const *grads, int flags, cudaStream_t stream,
                        int64_t lo = 0, int64_t count = -1, float *pre_slice = nullptr)
 {
+    const bool writes_pre = (flags & (kFirst | kRefresh)) && c->hp.local_updater == SSD_LOCAL_GLU;
+    // Merged device weights, pull iteration: the local update's result would be overwritten at once,
+    // so what remains is the server update and K stores of the new global weight, which is the
+    // server kernel's hand-over form ...
+    if (c->merged_dev && (flags & kPull) && !writes_pre) return launch_sync(c, grads, kCopy, stream, lo, count);
     StepParams p{};
     const bool shared = c->shared_pre || pre_slice;
     for (int i = 0; i < c->hp.K; ++i) {
@@ -552,6 +600,12 @@ ssd_status launch_step(ssd_ctx *c, const void *const *grads, int flags, cudaStre
     p.s = c->s;
     p.tt = table_of(c);
     p.tt.base = lo;
+    if (c->merged_dev && (flags & kPull)) {
+        // ... and with k = 1, where every pull also writes pre_weight, a kernel of its own
+        p.flags |= kMergedDev;
+        const Shape sh = sync_shape(c, max_vector(c, c->state32, grads, c->hp.K, lo, pre_slice), kCopy);
+        return p.tt.T ? launch_merged_pull_t<true>(c, p, sh, stream) : launch_merged_pull_t<false>(c, p, sh, stream);
+    }
     if (c->staging && ring_can_run(c, shared, lo, p.n)) return launch_step_ring(c, p, stream);
     const Shape sh = step_shape(c, flags, shared, max_vector(c, c->state32, grads, c->hp.K, lo, pre_slice), p.n);
     return p.tt.T ? launch_step_t<true>(c, p, sh, stream) : launch_step_t<false>(c, p, sh, stream);
@@ -655,11 +709,17 @@ ssd_status ssd_init(ssd_ctx **out, const ssd_layout *layout, const ssd_hparams *
     // values, every worker takes it from the same pulled global weight).
     bool shared_pre = device_pre && hp->K > 1 && b->pre[0] != nullptr;
     for (int i = 1; shared_pre && i < hp->K; ++i) shared_pre = b->pre[i] == b->pre[0];
+    // w_dev[i] == w_loc[i] for every worker: the device weights are the local weights themselves.
+    // It has to hold for all workers or for none.
+    int merged = 0;
+    for (int i = 0; workers && i < hp->K; ++i) merged += (b->w_dev[i] && b->w_dev[i] == b->w_loc[i]) ? 1 : 0;
+    const bool merged_dev = workers && merged == hp->K;
+    if (merged != 0 && !merged_dev) st = SSD_ERR_ARG;
     std::vector<const void *> all{b->w, b->mom};
     for (int i = 0; workers && i < hp->K; ++i) {
         all.push_back(b->w_loc[i]);
         if (device_pre && (!shared_pre || i == 0)) all.push_back(b->pre[i]);
-        all.push_back(b->w_dev[i]);
+        if (!merged_dev) all.push_back(b->w_dev[i]);
     }
     for (const void *p : all) {
         if (!p) st = SSD_ERR_ARG;
@@ -697,6 +757,7 @@ ssd_status ssd_init(ssd_ctx **out, const ssd_layout *layout, const ssd_hparams *
     c->has_workers = workers;
     c->shared_pre = shared_pre;
     c->pre_on_device = device_pre;
+    c->merged_dev = merged_dev;
     c->state32 = true;
     for (const void *p : all) c->state32 = c->state32 && aligned32(p);
     for (int i = 0; workers && i < hp->K; ++i) {
@@ -883,7 +944,8 @@ ssd_status ssd_step_host(ssd_ctx *ctx, const void *const *host_grads, void *cons
     // one of the device slices before the chunk's kernel (not on the first GLU call, which does
     // not read it) and copied back after it on the iterations that overwrite it.
     const bool host_pre = glu_stage && ctx->host_pre;
-    const bool pre_in = host_pre && !(flags & SSD_FLAG_FIRST);
+    // (nor on a pull iteration of a context with merged device weights, which skips the local update)
+    const bool pre_in = host_pre && !(flags & SSD_FLAG_FIRST) && !(ctx->merged_dev && (flags & SSD_FLAG_PULL));
     const bool pre_out = host_pre && (flags & (SSD_FLAG_FIRST | SSD_FLAG_REFRESH));
     const int slots = ctx->pre_slots;
 
@@ -1001,7 +1063,7 @@ ssd_status ssd_worker_weights(const ssd_ctx *ctx, int32_t worker, const float **
         int32_t stage, flags;
         schedule_of(ctx, ctx->iter - 1, &stage, &flags);
         if (stage == SSD_STAGE_WARMUP) v = (flags & SSD_FLAG_COPY) ? SSD_VIEW_LOCAL : SSD_VIEW_GLOBAL;
-        else v = (flags & SSD_FLAG_PULL) ? SSD_VIEW_DEVICE : SSD_VIEW_LOCAL;
+        else v = ((flags & SSD_FLAG_PULL) && !ctx->merged_dev) ? SSD_VIEW_DEVICE : SSD_VIEW_LOCAL;
     }
     if (view) *view = v;
     if (weights)

@@ -72,19 +72,22 @@ class DeviceState:
     shared_pre: one pre_weight arena for all workers.  host_pre: pre_weight lives in ONE pinned
     host arena and is streamed through `pre_slots` device slices by ssd_step_host (the other
     delay-stage calls are then not available); `host_chunk` sets the chunk of that pipeline.
+    merged_dev: no separate device weights (w_dev[i] is w_loc[i]; K arenas less).
     """
 
     def __init__(self, numels: Sequence[int], hp: B.ssd_hparams, w0: torch.Tensor,
                  device="cuda", fill: float = float("nan"), worker_state: bool = True,
                  shared_pre: bool = False, host_pre: bool = False, pre_slots: int = 2,
-                 host_chunk: int = 0):
+                 host_chunk: int = 0, merged_dev: bool = False):
         self.numels = [int(n) for n in numels]
         self.n = B.ssd_arena_numel(self.numels)
         assert w0.numel() == self.n and w0.dtype == torch.float32
         self.K = hp.K
         self.device = torch.device(device)
         n_pre = 0 if (not worker_state or host_pre) else (1 if shared_pre else self.K)
-        self.slab = ArenaSlab(2 + (2 * self.K if worker_state else 0) + n_pre, self.n, torch.float32, self.device)
+        self.merged_dev = bool(merged_dev and worker_state)
+        n_workers = 0 if not worker_state else (self.K if merged_dev else 2 * self.K)
+        self.slab = ArenaSlab(2 + n_workers + n_pre, self.n, torch.float32, self.device)
         arenas = self.slab.arenas
         self.slabs = [self.slab]
         self.w, self.mom = arenas[0], arenas[1]
@@ -98,11 +101,11 @@ class DeviceState:
             return
         # Algorithm 1 starts with every worker pulling w_0.
         self.w_loc = arenas[2:2 + self.K]
-        self.w_dev = arenas[2 + self.K:2 + 2 * self.K]
+        self.w_dev = self.w_loc if merged_dev else arenas[2 + self.K:2 + 2 * self.K]
+        for t in arenas[2 + self.K:]:
+            t.fill_(fill)
         for t in self.w_loc:
             t.copy_(self.w)
-        for t in self.w_dev + arenas[2 + 2 * self.K:]:
-            t.fill_(fill)
         if host_pre:
             self.host_pre = torch.full((self.n,), fill, dtype=torch.float32).pin_memory()
             self.pre = [self.host_pre] * self.K
@@ -116,7 +119,7 @@ class DeviceState:
             self.ctx.ssd_set_host_pre_weight(self.host_pre, self.pre_slices, pre_slots)
             return
         # shared_pre: one pre_weight buffer for all workers (K references to the same tensor)
-        self.pre = arenas[2 + 2 * self.K:] * (self.K if shared_pre else 1)
+        self.pre = arenas[2 + n_workers:] * (self.K if shared_pre else 1)
         self.ctx = B.Context(self.numels, hp, self.w, self.mom, self.w_loc, self.pre, self.w_dev)
 
     def worker_weights(self, i: int) -> torch.Tensor:
@@ -131,7 +134,7 @@ class DeviceState:
     def bytes(self) -> int:
         """Device bytes of the state arenas (and of the slices of a host-resident pre_weight)."""
         device_pre = {t.data_ptr() for t in self.pre if t.is_cuda}
-        total = (2 + len(self.w_loc) + len(device_pre) + len(self.w_dev)) * self.n * 4
+        total = (2 + len(self.w_loc) + len(device_pre) + (0 if self.merged_dev else len(self.w_dev))) * self.n * 4
         if len(self.slabs) > 1:
             total += self.pre_slices.numel() * 4
         return total

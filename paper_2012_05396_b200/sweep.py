@@ -7,6 +7,9 @@ launches, median and minimum reported):
     sync    ssd_server_sync_update               K*sg + 16 bytes per parameter
     glu     ssd_worker_glu_update, plain flags   sg + 12 bytes per parameter and worker
     step    ssd_step in the steps-delay stage    K*(sg+12) + 16 (+4K on refresh, +4K on pull)
+    step_merged  the same for a context without separate device weights: only its pull iterations
+            differ (server update + K stores of the new global weight, K*(sg+4) + 16) and only they
+            are reported
 and prints one JSON object per point.  State and gradients are uniform(-1,1) from the seeded
 generators.  Points whose footprint is below 1 GB rotate over several independent buffer sets (at
 least 1 GB together), so that a launch never finds its data in the 126 MB L2 left by the previous
@@ -157,13 +160,15 @@ def point(log2n: int, K: int, dtype: str, kernels, reps: int, peak: float, threa
             del st, grads
         else:
             skip("glu", fp)
-    if "step" in kernels:
-        fp = (2 + 3 * K) * n * 4 + K * n * sg
+    for merged in (False, True):
+        if ("step_merged" if merged else "step") not in kernels:
+            continue
+        fp = (2 + (2 if merged else 3) * K) * n * 4 + K * n * sg
         R = copies(fp)
         if _fits(fp * R):
             sets = []
             for _ in range(R):
-                st = DeviceState(numels, _hp(K, 4, dtype), w0, fill=0.0)
+                st = DeviceState(numels, _hp(K, 4, dtype), w0, fill=0.0, merged_dev=merged)
                 tune(st)
                 grads = _grads(n, K, dtype)
                 st.ctx.ssd_step(grads)                               # first GLU call
@@ -185,10 +190,14 @@ def point(log2n: int, K: int, dtype: str, kernels, reps: int, peak: float, threa
             for flags, ms in sorted(per_flag.items()):
                 b = K * (sg + 12) + 16 + (4 * K if flags & 2 else 0) + (4 * K if flags & 4 else 0)
                 name = "step" + ("+refresh" if flags & 2 else "") + ("+pull" if flags & 4 else "")
+                if merged:
+                    if not flags & 4:
+                        continue                                     # the other iterations are the plain form's
+                    b, name = K * (sg + 4) + 16, "step+pull (merged device weights)"
                 emit(name, fp, b * n, statistics.median(ms), min(ms))
             del sets
         else:
-            skip("step", fp)
+            skip("step_merged" if merged else "step", fp)
     torch.cuda.empty_cache()
     return out
 
@@ -198,7 +207,7 @@ def main():
     ap.add_argument("--log2n", type=int, nargs="+", default=[16, 18, 20, 22, 24, 26, 28])
     ap.add_argument("--K", type=int, nargs="+", default=[1, 4, 16, 32])
     ap.add_argument("--dtype", nargs="+", default=["f32", "bf16"], choices=["f32", "bf16"])
-    ap.add_argument("--kernels", nargs="+", default=["sync", "glu", "step"], choices=["sync", "glu", "step"])
+    ap.add_argument("--kernels", nargs="+", default=["sync", "glu", "step"], choices=["sync", "glu", "step", "step_merged"])
     ap.add_argument("--reps", type=int, default=20)
     ap.add_argument("--peak", type=float, default=0.0,
                     help="HBM copy rate in GB/s for the 'of measured' column (0 = read MEASURED_PEAKS.json, "

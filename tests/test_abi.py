@@ -299,6 +299,30 @@ def test_overlapping_buffers_are_rejected():
     assert e.value.status == B.SSD_ERR_ARG
 
 
+def test_merged_device_weights_are_all_or_none():
+    # w_dev[i] == w_loc[i] for every worker: accepted, and the view after a pull is the local weight;
+    # for some workers only, or a w_dev that merely overlaps a w_loc: rejected
+    K, W, k = 3, 1, 2
+    hp = B.make_hparams(K, 0.1, 0.9, W, k)
+    n = 1 << 12
+    w, mom, wl, pre, wdv = fake_ptrs(K)
+    ctx = B.Context([n], hp, w, mom, wl, pre, list(wl))
+    for it in range(7):
+        stage, flags = ctx.ssd_schedule(it)
+        ctx.ssd_advance()
+        p, view = ctx.ssd_worker_weights(2)
+        want = B.SSD_VIEW_GLOBAL if stage == B.SSD_STAGE_WARMUP and not flags & B.SSD_FLAG_COPY else B.SSD_VIEW_LOCAL
+        assert (p, view) == ((w, wl[2])[view], want)
+    for bad in ([wl[0], wdv[1], wdv[2]], [wdv[0], wdv[1], wl[2]], [wl[1], wl[0], wl[2]], [wl[0] + 16, wdv[1], wdv[2]]):
+        with pytest.raises(B.SsdError) as e:
+            B.Context([n], hp, w, mom, wl, pre, bad)
+        assert e.value.status == B.SSD_ERR_ARG
+    # a gradient may not reach into the merged buffers either
+    with pytest.raises(B.SsdError) as e:
+        ctx.ssd_step([wl[0] + 64, wdv[1], wdv[2]])
+    assert e.value.status == B.SSD_ERR_ARG and ctx.ssd_kernel_launches() == 0
+
+
 def test_host_pre_weight_mode_is_validated():
     K, n = 2, 4096
     hp = B.make_hparams(K, 0.1, 0.9, 0, 2)

@@ -371,6 +371,38 @@ def test_pull_and_pre_weight_invariants():
                 assert any(not np.array_equal(w_loc[i], w_loc[0]) for i in range(1, K))
 
 
+def test_device_weights_are_an_output_nothing_reads():
+    # Algorithm 1 broadcasts the local update's result to the devices and, on a pull iteration,
+    # overwrites the local weight right after.  Nothing in the method reads the device weights back,
+    # so scrambling them after every iteration must leave w, mom, every local weight and every
+    # pre_weight untouched.  (This is what lets a caller keep ONE buffer per worker for both: the
+    # result of a pull iteration's local update is then simply never produced.)
+    rng = np.random.default_rng(21)
+    K, N, T = 3, 17, 26
+    w0 = rng.standard_normal(N).astype(f32)
+    for W, k in ((0, 1), (2, 1), (1, 3), (4, 4)):
+        hp = Hyper(K=K, lr=0.1, m=0.9, W=W, k=k, wd=0.01)
+        stream = [rng_grads(rng, K, N, 1e-2) for _ in range(T)]
+        _, clean = run_config(hp, w0, stream)
+        st = State(hp, w0)
+        pulls = 0
+        for n, gs in enumerate(stream):
+            stage, flags = st.step(gs)
+            if stage == STAGE_DELAY and flags & F_PULL:
+                pulls += 1
+                for i in range(K):                       # on a pull the two differ: GLU result vs pulled weight
+                    assert not np.array_equal(st.w_dev[i], st.w_loc[i])
+            for i in range(K):
+                st.w_dev[i][:] = rng.standard_normal(N).astype(f32)
+            _, _, _, w, mom, w_loc, pre = clean[n]
+            np.testing.assert_array_equal(st.w, w)
+            np.testing.assert_array_equal(st.mom, mom)
+            for i in range(K):
+                np.testing.assert_array_equal(st.w_loc[i], w_loc[i])
+                np.testing.assert_array_equal(st.pre[i], pre[i])
+        assert pulls >= 3
+
+
 def test_zero_delay_reduces_to_ssgd():
     rng = np.random.default_rng(8)
     K, N, T = 2, 9, 10
