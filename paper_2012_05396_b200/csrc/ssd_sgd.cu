@@ -234,8 +234,13 @@ Shape sync_shape(const ssd_ctx *c, int max_vw, int flags = 0)
         // stage, and every pull of a context with merged device weights): 44 % of the traffic is
         // writes, and 384 threads per SM is the optimum whatever K (6.5-6.65 TB/s float32,
         // 6.25-6.5 bfloat16, against 5.9-6.1 with the shapes below)
-        const bool wide = c->hp.grad_dtype == SSD_BF16 && max_vw >= 16;
-        return finish_shape(c, wide ? Shape{16, 2, 128, 3} : Shape{8, 4, 128, 3}, max_vw, 8);
+        // (with one to three float32 workers there are too few streams for that: vectors of 16, or 512
+        // threads per SM for two workers, bring 5.2-6.2 TB/s to 6.4-6.6)
+        const bool bf16 = c->hp.grad_dtype == SSD_BF16;
+        Shape copy_shape = Shape{8, 4, 128, 3};
+        if (max_vw >= 16 && (bf16 || K == 1 || K == 3)) copy_shape = Shape{16, 2, 128, 3};
+        else if (!bf16 && K == 2) copy_shape = Shape{8, 2, 128, 4};
+        return finish_shape(c, copy_shape, max_vw, 8);
     }
     // (the batch is an upper bound: the K workers go in ceil(K / batch) batches of equal size)
     if (c->hp.grad_dtype == SSD_BF16) {

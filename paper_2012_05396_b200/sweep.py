@@ -196,6 +196,7 @@ def point(log2n: int, K: int, dtype: str, kernels, reps: int, peak: float, threa
                     b, name = K * (sg + 4) + 16, "step+pull (merged device weights)"
                 emit(name, fp, b * n, statistics.median(ms), min(ms))
             del sets
+            st = grads = None                                        # the loop variables still held the last set
         else:
             skip("step_merged" if merged else "step", fp)
     torch.cuda.empty_cache()
