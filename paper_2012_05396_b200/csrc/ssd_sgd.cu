@@ -281,6 +281,19 @@ Shape step_shape(const ssd_ctx *c, int flags, bool shared_pre, int max_vw, int64
         if (k_extra_stores && bf16) sh = Shape{16, 1, 128, 3};
         if (!k_extra_stores && (K == 1 || (K == 2 && !bf16))) sh = Shape{16, 1, 128, 3};
     }
+    // One shared pre_weight (also a slice of a host-resident one): K fewer read streams, so two
+    // workers' loads per thread keep as many bytes in flight; measured at 2^26 elements, K = 4..32:
+    // plain and refresh iterations +2.5 % (float32, K >= 8) and +4..8 % (bfloat16, which sat at 5.9-6.3
+    // TB/s before); pull iterations +2.7 % (float32) and +2..5 % (bfloat16, vectors of 8 again).
+    if (shared_pre && !sgd && K >= 4) {
+        if (!(flags & kPull)) {
+            if (bf16 || K >= 8) sh = Shape{8, 2, 128, 5};
+        } else if (bf16) {
+            sh = Shape{8, 1, 128, 5};
+        } else {
+            sh = K >= 8 ? Shape{8, 2, 128, 3} : Shape{16, 1, 128, 3};
+        }
+    }
     // A step whose whole traffic fits in L2 (ResNet-20/56 sized arenas) is bound by latency, not by
     // DRAM: smaller vectors spread it over more threads, and two workers' loads per thread halve the
     // number of dependent round trips.
