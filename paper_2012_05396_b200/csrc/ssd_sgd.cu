@@ -277,9 +277,12 @@ Shape step_shape(const ssd_ctx *c, int flags, bool shared_pre, int max_vw, int64
     const bool sgd = c->hp.local_updater == SSD_LOCAL_SGD;
     const bool k_extra_stores = (flags & kPull) || (!shared_pre && !sgd && (flags & (kRefresh | kFirst)));
     Shape sh = k_extra_stores ? Shape{8, 1, 128, 4} : Shape{8, 1, 128, 5};
+    // plain iterations with many workers: two workers' loads per thread at 512 threads per SM (+1.4 %)
+    if (!k_extra_stores && K >= 12) sh = Shape{8, 2, 128, 4};
     if (max_vw >= 16) {
         if (k_extra_stores && bf16) sh = Shape{16, 1, 128, 3};
         if (!k_extra_stores && (K == 1 || (K == 2 && !bf16))) sh = Shape{16, 1, 128, 3};
+        if (!k_extra_stores && K == 4 && !bf16) sh = Shape{16, 2, 128, 3};
     }
     // One shared pre_weight (also a slice of a host-resident one): K fewer read streams, so two
     // workers' loads per thread keep as many bytes in flight; measured at 2^26 elements, K = 4..32:
