@@ -252,11 +252,12 @@ Shape sync_shape(const ssd_ctx *c, int max_vw, int flags = 0)
         else if (K >= 5) sh = Shape{16, 8, 128, 3};
         else if (K == 4) sh = Shape{16, 4, 128, 3};
         else if (K == 3) sh = Shape{8, 4, 128, 6};
-        else if (K == 2) sh = Shape{16, 2, 128, 4};
+        else if (K == 2) sh = Shape{16, 1, 128, 6};
         else sh = Shape{16, 1, 128, 4};
         if (max_vw < 16) sh = K >= 3 ? Shape{8, 4, 128, 6} : Shape{8, 1, 128, K == 1 ? 4 : 6};
     } else {
-        if (K >= 8 || K == 4) sh = Shape{8, 4, 128, 5};
+        if (K == 4) sh = Shape{8, 4, 256, 3};
+        else if (K >= 8) sh = Shape{8, 4, 128, 5};
         else if (K >= 5) sh = Shape{8, 8, 128, 4};
         else if (K == 3) sh = Shape{16, 4, 128, 3};
         else if (K == 2) sh = Shape{16, 2, 128, 3};
