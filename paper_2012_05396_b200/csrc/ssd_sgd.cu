@@ -298,6 +298,14 @@ Shape step_shape(const ssd_ctx *c, int flags, bool shared_pre, int max_vw, int64
             sh = K >= 8 ? Shape{8, 2, 128, 3} : Shape{16, 1, 128, 3};
         }
     }
+    // Plain-SGD local updater: no pre_weight streams either.  Pull iterations are half writes: 384
+    // threads per SM with two workers' loads per thread (float32, +2.3 %), vectors of 8 at 640 threads
+    // per SM (bfloat16: 6.3-6.4 TB/s against 5.7-5.9 with the vectors of 16 of the GLU form); the other
+    // iterations with bfloat16 gradients and few workers want two workers' loads per thread (+5 %).
+    if (sgd && K >= 4) {
+        if (flags & kPull) sh = bf16 ? Shape{8, 1, 128, 5} : Shape{8, 2, 128, 3};
+        else if (bf16 && K < 12) sh = Shape{8, 2, 128, 5};
+    }
     // A step whose whole traffic fits in L2 (ResNet-20/56 sized arenas) is bound by latency, not by
     // DRAM: smaller vectors spread it over more threads, and two workers' loads per thread halve the
     // number of dependent round trips.
@@ -625,7 +633,11 @@ ssd_status launch_step(ssd_ctx *c, const void *const *grads, int flags, cudaStre
     if (c->merged_dev && (flags & kPull)) {
         // ... and with k = 1, where every pull also writes pre_weight, a kernel of its own
         p.flags |= kMergedDev;
-        const Shape sh = sync_shape(c, max_vector(c, c->state32, grads, c->hp.K, lo, pre_slice), kCopy);
+        // K more loads than the hand-over form (the old local weights): vectors of 16, more loads per batch
+        // (6.5-6.6 TB/s at 2^26 elements against 5.7 float32 / 6.25 bfloat16 with the hand-over shape)
+        const int max_vw = max_vector(c, c->state32, grads, c->hp.K, lo, pre_slice);
+        const Shape wide = c->hp.grad_dtype == SSD_BF16 ? Shape{16, 8, 128, 3} : Shape{16, 4, 128, 4};
+        const Shape sh = max_vw >= 16 ? finish_shape(c, wide, max_vw, 8) : sync_shape(c, max_vw, kCopy);
         return p.tt.T ? launch_merged_pull_t<true>(c, p, sh, stream) : launch_merged_pull_t<false>(c, p, sh, stream);
     }
     if (c->staging && ring_can_run(c, shared, lo, p.n)) return launch_step_ring(c, p, stream);
