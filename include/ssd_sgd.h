@@ -244,7 +244,9 @@ ssd_status ssd_server_sync_update_static(ssd_ctx *ctx, const void *const *grads,
  *     else:       w_loc_i[j] = r
  * `flags` is any combination of SSD_FLAG_FIRST / REFRESH / PULL.  With PULL, `w`
  * must already hold this iteration's server result (enqueue the server update
- * first on the same stream).  Does not read or move the counters.  Errors:
+ * first on the same stream).  For a context with merged device weights a PULL call
+ * reduces to: if FIRST or REFRESH: pre_i[j] = w_loc_i[j]; then w_loc_i[j] = w[j].
+ * Does not read or move the counters.  Errors:
  * SSD_ERR_ARG (worker out of range, unknown flag, NULL grad), SSD_ERR_STATE
  * (delay_k == 0: there is no delay stage), SSD_ERR_ALIGN.  One kernel launch. */
 ssd_status ssd_worker_glu_update(ssd_ctx *ctx, int32_t worker, const void *grad, int32_t flags,

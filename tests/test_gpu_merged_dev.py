@@ -29,7 +29,7 @@ def flat_layout(numels):
 
 
 def run_merged(lay, K, W, k, iters, mode, bf16=False, wd=1e-3, shared_pre=False, local_sgd=False,
-               per_tensor=False, shape=None, check_every=1):
+               per_tensor=False, shape=None, check_every=1, staging=0):
     ohp, chp = make_hp(K, 0.1, 0.9, W, k, wd=wd, bf16=bf16, local_sgd=local_sgd)
     w0 = synth.init_weights(lay)
     dev = DeviceState(lay.numels, chp, w0, merged_dev=True, shared_pre=shared_pre)
@@ -43,6 +43,8 @@ def run_merged(lay, K, W, k, iters, mode, bf16=False, wd=1e-3, shared_pre=False,
         dev.ctx.ssd_set_tensor_scales(lr_mult, wd_mult, table)
     if shape:
         dev.ctx.ssd_set_kernel_shape(*shape)
+    if staging:
+        dev.ctx.ssd_set_staging(staging)
     ref = oracle.State(ohp, w0.numpy())
     mask = synth.valid_mask(lay, "cuda")
     seen = 0
@@ -83,6 +85,14 @@ def test_merged_device_weights_shared_pre_weight_and_plain_sgd():
     run_merged(lay, 4, 2, 3, 10, "fused", shared_pre=True)
     run_merged(lay, 4, 1, 2, 8, "fused", local_sgd=True)
     run_merged(lay, 3, 0, 1, 5, "split", local_sgd=True)
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_merged_device_weights_with_the_staged_fused_step(bf16):
+    # the shared-memory ring runs the iterations without a pull; the pulls stay on the register path
+    lay = flat_layout([70001, 12, 4099])
+    dev, _, seen = run_merged(lay, 3, 1, 3, 9, "fused", bf16=bf16, staging=3)
+    assert seen & 7 == 7 and dev.ctx.ssd_staging_error() == 0
 
 
 @pytest.mark.parametrize("bf16", [False, True])

@@ -485,11 +485,14 @@ def test_layer_by_layer_stepping_equals_one_step(bf16):
     for i, cnt in enumerate((5, 1, 10, 3, 64, 7, 1024, 2, 36, 4100, 12, 9, 20000, 4, 4, 33)):
         lay.add(f"x{i}", cnt, "he" if i % 3 else "zero", 16)
     T = lay.num_tensors
-    _, chp = make_hp(K, 0.1, 0.9, W, k, wd=1e-3, bf16=bf16)
+    ohp, chp = make_hp(K, 0.1, 0.9, W, k, wd=1e-3, bf16=bf16)
     w0 = synth.init_weights(lay)
     whole = DeviceState(lay.numels, chp, w0, shared_pre=True)
     layered = DeviceState(lay.numels, chp, w0, shared_pre=True)
     wd_mult = [1.0 if kind == "he" else 0.0 for kind in lay.kinds]
+    ends = [lay.offsets[t + 1] if t + 1 < T else lay.padded_numel for t in range(T)]
+    ohp.set_tensor_scales(ends, [1.0] * T, wd_mult)
+    ref = oracle.State(ohp, w0.numpy())                    # and both must equal the CPU oracle
     tables = [torch.empty(s.ctx.ssd_tensor_table_bytes(), dtype=torch.uint8, device="cuda") for s in (whole, layered)]
     whole.ctx.ssd_set_tensor_scales(None, wd_mult, tables[0])
     layered.ctx.ssd_set_tensor_scales(None, wd_mult, tables[1])
@@ -508,7 +511,9 @@ def test_layer_by_layer_stepping_equals_one_step(bf16):
         for first, count in reversed(groups):
             layered.ctx.ssd_step_tensors(grads, first, count)
         layered.ctx.ssd_advance()
+        ref.step([oracle_grad(g, bf16) for g in grads])
         torch.cuda.synchronize()
+        compare_states(layered, ref, f"layer groups, iter {n}")
         for name in ("w", "mom"):
             assert torch.equal(getattr(whole, name).view(torch.int32), getattr(layered, name).view(torch.int32)), (name, n)
         for i in range(K):
