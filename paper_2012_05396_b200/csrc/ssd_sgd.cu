@@ -537,8 +537,8 @@ ssd_status launch_step_t(ssd_ctx *c, StepParams &p, const Shape &sh, cudaStream_
     return bf16 ? launch_step_b<kBF16, 4, PT>(c, p, sh, stream) : launch_step_b<kF32, 4, PT>(c, p, sh, stream);
 }
 
-// Pull iteration that also writes pre_weight (k = 1) of a context with merged device weights; the
-// loads are the server kernel's, so it takes the server kernel's shape and batches.
+// Pull iteration that also writes pre_weight (k = 1) of a context with merged device weights.  Its
+// gradient loads are batched like the server kernel's (the same limits on loads in flight).
 template <int GT, int VW, bool PT>
 ssd_status launch_merged_pull_b(ssd_ctx *c, StepParams &p, const Shape &sh, cudaStream_t stream)
 {

@@ -8,7 +8,6 @@ must equal it bit for bit on every iteration (compare_states leaves out only w_d
 """
 import itertools
 
-import numpy as np
 import pytest
 import torch
 
